@@ -273,14 +273,11 @@ def test_anchor_position_matters_and_may_be_ahead():
 
 
 def test_token_permutation_inside_a_frame_changes_nothing_but_order():
-    """Keys are a set: permuting the tokens of the chunk (with their positions, i.e. comparing outputs row by
-    row after undoing the permutation of the queries) is only visible through the positions."""
+    """Keys are a set: with the positions taken out of play (a huge rotary base leaves only pair 0 of each axis
+    turning, and those input dims are zeroed) permuting the chunk's keys together with their values changes
+    nothing."""
     w = W.scaled(TINY, anchor_policy="none", grid_h=1, grid_w=16)
-    orc = make_oracle(w, O.F32)
     q, k, v = (t.numpy() for t in W.qkv(w, 6, 0, 0, 0, 1, torch.float32))
-    st, base = orc.chunk_forward(0, 0, 0, 1, 0, q, k, v)
-    # same tokens, K/V of all tokens made position-free by zero rotation: use theta so that only pair 0 turns,
-    # and zero those input dims -> then key order cannot matter
     for arr in (q, k):
         arr[..., 0:2] = 0
         arr[..., 24:26] = 0
@@ -291,7 +288,156 @@ def test_token_permutation_inside_a_frame_changes_nothing_but_order():
     orc_b = make_oracle(w, O.F32, rope_theta=1e300)
     st, b = orc_b.chunk_forward(0, 0, 0, 1, 0, q, k[perm], v[perm])
     assert np.allclose(a, b, atol=1e-6)
-    assert base.shape == a.shape
+
+
+def _strided_positions(n_frames, first, stride, grid_h, grid_w):
+    """[n_frames*grid_h*grid_w, 1, 3] positions of a block whose frames sit at first + f*stride (built here, not
+    taken from the oracle or from paper_defs.token_positions, which only knows dense chunks)."""
+    pos = [(first + f * stride, y, x) for f in range(n_frames) for y in range(grid_h) for x in range(grid_w)]
+    return np.asarray(pos, dtype=np.int64)[:, None, :]
+
+
+def test_order_of_visible_segments_does_not_matter():
+    """The visible keys are a set (the licence to read the banks in physical slot order): (a) the oracle, which
+    concatenates [anchors | history | own] in that order, equals the textbook softmax over the same keys gathered
+    in the opposite order [own | history newest first | anchors reversed]; (b) handing the oracle its anchor
+    slots in another order changes the output only by summation rounding."""
+    w = W.scaled(TINY, grid_h=3, grid_w=4, n_anchor_slots=2, visible_anchors=2, anchor_policy="none", total_frames=4)
+    anchors = {}
+    orcs = [make_oracle(w, O.F32) for _ in range(2)]
+    for slot, fpos in ((0, 9), (1, 2)):
+        k, v = (t.numpy() for t in W.anchor_kv(w, 21, slot, 0, torch.float32))
+        anchors[slot] = (k, v, fpos)
+        for orc in orcs:
+            assert orc.anchor_publish(slot, fpos, 0, k, v) == O.OK
+    calls = []
+    for i in range(w.n_chunks):
+        q, k, v = (t.numpy() for t in W.qkv(w, 21, i, 0, 0, 1, torch.float32))
+        calls.append((q, k, v))
+        st, out_fwd = orcs[0].chunk_forward(0, 0, i, 1, i, q, k, v, [0, 1])
+        st2, out_rev = orcs[1].chunk_forward(0, 0, i, 1, i, q, k, v, [1, 0])
+        assert st == O.OK and st2 == O.OK and orcs[0].advance(0) == O.OK and orcs[1].advance(0) == O.OK
+        assert np.allclose(out_fwd, out_rev, atol=1e-6)
+        ks, vs = [], []
+        for j in range(i, max(0, i - w.history_chunks) - 1, -1):          # own first, then history newest first
+            pos = P.token_positions(1, j, w.grid_h, w.grid_w)[:, None, :]
+            ks.append(P.rope_complex(calls[j][1], pos))
+            vs.append(calls[j][2].astype(np.float64))
+        for slot in (1, 0):                                               # anchors last, reversed
+            ak, av, fpos = anchors[slot]
+            ks.append(P.rope_complex(ak, P.token_positions(1, fpos, w.grid_h, w.grid_w)[:, None, :]))
+            vs.append(av.astype(np.float64))
+        K, V = np.concatenate(ks), np.concatenate(vs)
+        Q = P.rope_complex(q, P.token_positions(1, i, w.grid_h, w.grid_w)[:, None, :])
+        for h in range(w.n_heads):
+            assert np.allclose(out_fwd[:, h], P.softmax_attention(Q[:, h], K[:, h], V[:, h]), atol=2e-5), (i, h)
+
+
+def test_identical_keys_across_all_segments_return_the_mean_of_all_visible_values():
+    """Zero keys in the anchors, in every history chunk and in the own chunk: every score is 0, so the output is
+    the plain mean of V over anchor + history + own rows - and only over those (the evicted chunk's values
+    must not enter)."""
+    w = W.scaled(TINY, grid_h=2, grid_w=4, total_frames=5, anchor_policy="none", n_anchor_slots=2, visible_anchors=2)
+    orc = make_oracle(w, O.BF16)
+    avs = []
+    for slot, fpos in ((0, 7), (1, 3)):
+        k, v = (t.float().numpy() for t in W.anchor_kv(w, 33, slot, 0))
+        avs.append(v)
+        assert orc.anchor_publish(slot, fpos, 0, np.zeros_like(k), v) == O.OK
+    vs = []
+    for i in range(w.n_chunks):
+        q, k, v = (t.float().numpy() for t in W.qkv(w, 33, i, 0, 0, 1))
+        vs.append(v)
+        st, out = orc.chunk_forward(0, 0, i, 1, i, q, np.zeros_like(k), v, [0, 1])
+        assert st == O.OK and orc.advance(0) == O.OK
+        visible = np.concatenate(avs + vs[max(0, i - w.history_chunks):i + 1]).astype(np.float64)
+        want = visible.mean(axis=0, keepdims=True).repeat(len(q), 0)
+        assert np.allclose(out, want, atol=1e-6), i
+        if i > w.history_chunks:   # the chunk that left the window would have moved the mean
+            with_evicted = np.concatenate(avs + vs[i - w.history_chunks - 1:i + 1]).astype(np.float64).mean(axis=0)
+            assert np.abs(with_evicted - want[0]).max() > 1e-3
+
+
+# ----------------------------------------------------------------------------- planner side (Alg. 1 Phase A)
+
+def _planner_workload():
+    # blocks of B_P = 3 anchor latents that lie Delta = 10 positions apart, H_P = 6 earlier blocks visible
+    return W.scaled(W.PAPER_480P_PLANNER, n_layers=1, n_heads=2, head_dim=64, grid_h=2, grid_w=3)
+
+
+@pytest.mark.parametrize("dtype", [O.F32, O.BF16])
+def test_planner_blocks_sit_at_the_anchor_positions_of_the_worked_example(dtype):
+    """Blocks of anchor latents (frame f of block j at 30 j + 10 f: the worked example's {0,10,20}, {30,40,50},
+    {60,70,80}) through an oracle with frame stride 10, every call against the textbook softmax over keys
+    rotated at positions written out here."""
+    import json, os
+    gold = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "paper_values.json")))["worked_example"]
+    w = _planner_workload()
+    delta = w.frame_pos_stride
+    assert delta == gold["delta"] == 10 and w.chunk_frames == gold["B_P"] == 3
+    orc = make_oracle(w, dtype, frame_pos_stride=delta)
+    blocks = []
+    worst = 0.0
+    for j in range(3):
+        first = j * w.chunk_frames * delta
+        frames = [first + f * delta for f in range(w.chunk_frames)]
+        assert frames == gold["anchor_positions"][3 * j:3 * j + 3]
+        q, k, v = W.qkv(w, 11, j, 0, 0, w.chunk_frames, tdtype(dtype))
+        st, out = orc.chunk_forward(0, 0, j, w.chunk_frames, first, q.float().numpy(), k.float().numpy(),
+                                    v.float().numpy())
+        assert st == O.OK and orc.advance(0) == O.OK
+        pos = _strided_positions(w.chunk_frames, first, delta, w.grid_h, w.grid_w)
+        blocks.append((P.rope_complex(k.float().numpy(), pos), v.double().numpy()))
+        K = np.concatenate([b[0] for b in blocks])
+        V = np.concatenate([b[1] for b in blocks])
+        Q = P.rope_complex(q.float().numpy(), pos)
+        for h in range(w.n_heads):
+            want = P.softmax_attention(Q[:, h], K[:, h], V[:, h])
+            worst = max(worst, float(np.abs(out[:, h] - want).max()))
+        # the bank holds K rotated at the strided positions (a dense-chunk rotation would differ from frame 1 on)
+        ck, _ = orc.ring_slot(0, 0, j % (w.history_chunks + 1))
+        tol = 1e-5 if dtype == O.F32 else 2.0 ** -7
+        assert np.abs(ck - blocks[-1][0]).max() < tol
+        dense = P.rope_complex(k.float().numpy(), P.token_positions(w.chunk_frames, first, w.grid_h, w.grid_w)[:, None, :])
+        assert np.abs(ck - dense).max() > 0.1
+    assert worst < (2e-5 if dtype == O.F32 else 2e-2), worst
+
+
+def test_planner_republish_keeps_the_clean_endpoint_forward_and_never_reads_the_own_block_twice():
+    """Alg. 1 Phase A: S denoising forwards of block j, then one clean-endpoint forward whose K/V are what the
+    bank keeps.  Every one of the S+1 calls reads Tail_{H_P}(A) plus its OWN K/V (not the K/V an earlier forward of
+    the same block left in the slot), and after the last call the slot holds exactly that call's K'/V."""
+    w = _planner_workload()
+    S, delta = 4, w.frame_pos_stride
+    orc = make_oracle(w, O.F32, frame_pos_stride=delta)
+    kept = []      # per finished block: (rotated K of the clean-endpoint forward, its V)
+    for j in range(3):
+        first = j * w.chunk_frames * delta
+        pos = _strided_positions(w.chunk_frames, first, delta, w.grid_h, w.grid_w)
+        for f in range(S + 1):
+            q, k, v = (t.numpy() for t in W.qkv(w, 12, j, f, 0, w.chunk_frames, torch.float32))
+            st, out = orc.chunk_forward(0, 0, j, w.chunk_frames, first, q, k, v)
+            assert st == O.OK
+            own = (P.rope_complex(k, pos), v.astype(np.float64))
+            hist = kept[max(0, j - w.history_chunks):]
+            K = np.concatenate([b[0] for b in hist] + [own[0]])
+            V = np.concatenate([b[1] for b in hist] + [own[1]])
+            Q = P.rope_complex(q, pos)
+            for h in range(w.n_heads):
+                assert np.allclose(out[:, h], P.softmax_attention(Q[:, h], K[:, h], V[:, h]), atol=2e-5), (j, f, h)
+            ck, cv = orc.ring_slot(0, 0, j % (w.history_chunks + 1))
+            assert np.array_equal(cv, v) and np.abs(ck - own[0]).max() < 1e-5
+            assert orc.ring_state(0)["next_chunk"] == j      # still the same block until Tail is applied
+        kept.append(own)
+        assert orc.advance(0) == O.OK
+        # bit for bit: the slot equals a fresh oracle's publish of the last forward alone
+        solo = make_oracle(w, O.F32, frame_pos_stride=delta)
+        for jj in range(j):
+            z = np.zeros_like(k)
+            assert solo.chunk_forward(0, 0, jj, w.chunk_frames, 0, z, z, z, rows=[])[0] == O.OK and solo.advance(0) == O.OK
+        assert solo.chunk_forward(0, 0, j, w.chunk_frames, first, q, k, v, rows=[])[0] == O.OK
+        a, b = orc.ring_slot(0, 0, j % (w.history_chunks + 1)), solo.ring_slot(0, 0, j % (w.history_chunks + 1))
+        assert np.array_equal(a[0].view(np.uint32), b[0].view(np.uint32)) and np.array_equal(a[1], b[1])
 
 
 # ----------------------------------------------------------------------------- ring bookkeeping and isolation
