@@ -34,9 +34,28 @@ import ff_workloads as W  # noqa: E402
 WORKLOAD = "wan1p3b_480p"
 NOMINAL_BF16_TFLOPS = 2250.0
 N_IO = 8                 # distinct resident Q/K/V sets cycled over the layer-calls (345 MB > the 126 MB L2)
-CPU_SAMPLE_ROWS = 512    # query rows of one steady-state layer-call the oracle is timed on
-# DRAM bytes (read + write) one attention launch moved in the ncu capture summarised under profiles/
-NCU_TRAFFIC_BYTES_PER_ATTN_LAUNCH = 122.4e6  # mean of two captured launches (profiles/attn_tcgen05_wan1p3b_480p.md)
+CPU_SAMPLE_ROWS = 0      # query rows of one steady-state layer-call the oracle is timed on (0 = all of them)
+ATTN_KERNEL_SOURCE = os.path.join(ROOT, "paper_2609_32540_b200", "csrc", "attn_sm100.cu")
+ATTN_PROFILE = os.path.join(ROOT, "profiles", "attn_tcgen05_wan1p3b_480p.json")
+
+
+def blob_hash(path: str) -> str:
+    """The hash git gives a file's content (sha1 over a "blob <size>" header and the bytes)."""
+    import hashlib
+    data = open(path, "rb").read()
+    return hashlib.sha1(b"blob %d\0" % len(data) + data).hexdigest()
+
+
+def ncu_traffic(workload: str) -> dict:
+    """DRAM bytes per attention launch from the committed ncu summary of the headline workload, with a flag that
+    says whether the kernel source has changed since that capture (then the figure describes an older kernel)."""
+    if workload != WORKLOAD or not os.path.exists(ATTN_PROFILE):
+        return dict(traffic=None, traffic_source="no ncu capture of this workload")
+    prof = json.load(open(ATTN_PROFILE))
+    per_launch = prof["dram_bytes_read_per_launch"] + prof["dram_bytes_write_per_launch"]
+    return dict(traffic=per_launch, traffic_source=os.path.relpath(ATTN_PROFILE, ROOT),
+                traffic_stale=blob_hash(ATTN_KERNEL_SOURCE) != prof["kernel_source_blob"],
+                traffic_captured_on=prof.get("capture_case"))
 
 
 def read_peaks():
@@ -109,6 +128,13 @@ def whole_job_tflops(flops_per_rank: float, ms: float, world: int) -> float:
     return world * flops_per_rank / (ms * 1e-3) / 1e12
 
 
+def attn_algorithmic_bytes(w: W.Workload) -> float:
+    """HBM bytes one steady-state attention launch cannot avoid: rotated queries in, output out, every visible key
+    and value row once (bf16)."""
+    n_q = w.chunk_frames * w.tokens_per_frame
+    return 2.0 * w.n_heads * w.head_dim * (2 * n_q + 2 * w.steady_n_kv())
+
+
 def chunk_flops(w: W.Workload, i: int) -> float:
     """Exact attention flops of all S*Ly layer-calls of chunk i (only keys that are really visible)."""
     n_q = w.chunk_frames * w.tokens_per_frame
@@ -142,7 +168,8 @@ class OracleStream:
         """Returns (TFLOP/s, seconds) of one layer-call on n_rows sampled rows (n_rows = 0: publish only)."""
         w, i = self.w, self.chunk
         n_q = w.chunk_frames * w.tokens_per_frame
-        rows = [int(r * n_q / n_rows) for r in range(n_rows)]
+        rows = None if n_rows >= n_q else [int(r * n_q / n_rows) for r in range(n_rows)]
+        n_rows = min(n_rows, n_q)
         t0 = time.perf_counter()
         st, _ = self.orc.chunk_forward(0, 0, i, w.chunk_frames, i * w.chunk_frames, self.q, self.k, self.v, [0],
                                        rows=rows)
@@ -159,7 +186,7 @@ class OracleStream:
 def oracle_sample(w: W.Workload, n_rows: int):
     """One timed steady-state sample: (TFLOP/s, seconds, threads)."""
     s = OracleStream(w)
-    v, dt = s.step(n_rows)
+    v, dt = s.step(n_rows or w.chunk_frames * w.tokens_per_frame)
     return v, dt, s.threads()
 
 
@@ -383,10 +410,11 @@ def measure_wavefront(P, dev, local: int, workload: str, steps: int) -> dict:
     return out
 
 
-def measure_clip_at_once(P, dev, local: int, group: int = 8) -> dict:
+def measure_clip_at_once(P, dev, local: int, group: int = 27) -> dict:
     """Extra: one stage of a whole 81-latent clip at the paper's budget (H = 5, Gamma windows, 27 chunks) in the
     clip-at-once form: `group` consecutive chunks of the stage per batched launch under the chunk-wise causal
-    mask (bank with H + group slots), all layers."""
+    mask (bank with H + group slots), all layers.  group = 27 is the whole clip in ONE attention launch per
+    layer."""
     w = W.scaled(W.PAPER_480P, n_stages=1, n_anchor_slots=9)
     N = w.n_chunks
     cfg = P.make_config(n_layers=w.n_layers, n_heads=w.n_heads, head_dim=w.head_dim, grid_h=w.grid_h, grid_w=w.grid_w,
@@ -432,6 +460,68 @@ def measure_clip_at_once(P, dev, local: int, group: int = 8) -> dict:
     assert st == 0 and word == 0, (st, hex(word))
     out = dict(workload=w.name + ", one stage", chunks=N, group=group, layer_calls=N * w.n_layers, ms_per_clip_stage=ms,
                tflops=flops / (ms * 1e-3) / 1e12)
+    cache.close()
+    del arena, sets
+    torch.cuda.empty_cache()
+    return out
+
+
+def measure_peaked_logits(P, dev, local: int, workload: str, steps: int, logit_gain: float = 8.0) -> dict:
+    """Extra: the headline step on inputs whose logits are `logit_gain` times larger (peaked softmax).  The
+    attention kernel raises a row's reference maximum lazily and rescales its accumulator when it does, so its
+    speed depends on the data; the headline's RMS-normalised inputs hardly ever trigger that path, these do."""
+    base = W.CONFIGS[workload]
+    warm = base.history_chunks + 2
+    w = W.scaled(base, total_frames=(warm + steps + 2) * base.chunk_frames, clip_anchor_pos=False,
+                 max_frame_pos=(warm + steps + 12) * base.chunk_frames + 16)
+    cfg = P.make_config(n_layers=w.n_layers, n_heads=w.n_heads, head_dim=w.head_dim, grid_h=w.grid_h, grid_w=w.grid_w,
+                        chunk_frames=w.chunk_frames, n_stages=w.n_stages, history_chunks=w.history_chunks,
+                        n_anchor_slots=w.n_anchor_slots, max_visible_anchors=w.visible_anchors, dtype=P.FF_BF16,
+                        attn_impl=P.FF_ATTN_TCGEN05, max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta,
+                        device=local)
+    nbytes = P.ff_cache_query_bytes(cfg)
+    arena = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    cache = P.Cache(cfg, arena.data_ptr(), nbytes)
+    stream = torch.cuda.current_stream().cuda_stream
+    sets = []
+    for sidx in range(N_IO):
+        q, k, v = W.qkv(w, 5, sidx, 0, 0, logit_gain=logit_gain)
+        sets.append((q.to(dev), k.to(dev), v.to(dev), torch.empty_like(q, device=dev)))
+    io = P.make_io([(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr()) for q, k, v, o in sets])
+    ak, av = (t.to(dev) for t in W.anchor_kv(w, 5, 0, 0))
+    published = set()
+
+    def step(i):
+        ids = W.visible_anchor_ids(w, i)
+        for m in ids:
+            if m not in published:
+                published.add(m)
+                for l in range(w.n_layers):
+                    assert cache.ff_anchor_publish(W.anchor_slot(w, m), W.anchor_frame_pos(w, m), l, ak.data_ptr(),
+                                                   av.data_ptr(), stream) == 0
+        assert cache.ff_sched_run_chunk(i, w.chunk_frames, i * w.chunk_frames, [W.anchor_slot(w, m) for m in ids], io,
+                                        stream) == 0
+
+    for i in range(warm):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    flops = 0.0
+    for i in range(warm, warm + steps):
+        step(i)
+        flops += chunk_flops(w, i)
+    e1.record()
+    torch.cuda.synchronize()
+    st, word = cache.ff_cache_status(stream)
+    assert st == 0 and word == 0, (st, hex(word))
+    ms = e0.elapsed_time(e1)
+    # how peaked: share of a row's probability mass on its largest key, for a few rows of one head (diagnostic)
+    q, k = sets[0][0][:64, 0].float(), torch.cat([s_[1][:, 0].float() for s_ in sets[:3]])
+    p = torch.softmax(q @ k.T / w.head_dim ** 0.5, dim=-1)
+    out = dict(workload=workload, logit_gain=logit_gain, steps=steps, ms_per_step=ms / steps,
+               tflops=flops / (ms * 1e-3) / 1e12, chunks_per_s=steps / (ms * 1e-3),
+               mean_top1_probability_unrotated_sample=float(p.max(dim=-1).values.mean()))
     cache.close()
     del arena, sets
     torch.cuda.empty_cache()
@@ -686,11 +776,13 @@ def run_gpu(args):
                   h2d_bytes_per_step=3 * call_bytes * n_calls, d2h_bytes_per_step=call_bytes * n_calls,
                   steps=args.e2e_steps, ms_per_step=e2e_ms / args.e2e_steps) if e2e_ms else None),
         gpu_launches=launches,
-        roofline=dict(bound="tensor", kernel="attn_tcgen05_kernel<128, false> (+ attn_combine_kernel<128>)", achieved=attn_tflops, peak=peaks["sustained"],
+        roofline=dict(bound="tensor", kernel=f"attn_tcgen05_kernel<{w.head_dim}, false, false> (+ attn_combine_kernel<{w.head_dim}, false>)",
+                      achieved=attn_tflops, peak=peaks["sustained"],
                       unit="TFLOP/s", frac=attn_tflops / peaks["sustained"], frac_of_burst_peak=attn_tflops / peaks["burst"],
                       peak_source=f"{peaks['source']} bf16 GEMM, sustained (kernel timed inside a long step)",
                       ms_per_launch=attn_ms, launches_timed=prof["attn_launches"],
-                      flops_per_launch=attn_flops_per_launch, traffic=NCU_TRAFFIC_BYTES_PER_ATTN_LAUNCH,
+                      flops_per_launch=attn_flops_per_launch, **ncu_traffic(args.workload),
+                      algorithmic_bytes_per_launch=attn_algorithmic_bytes(w),
                       publish=dict(bound="hbm", achieved=publish_gbs, peak=peaks["hbm_gbs"], unit="GB/s",
                                    frac=publish_gbs / peaks["hbm_gbs"], ms_per_launch=publish_ms,
                                    bytes_per_launch=publish_bytes)),
@@ -706,14 +798,17 @@ def run_gpu(args):
         line["paper_budget"] = measure_paper_budget(P, dev, local)
         line["adjacent_steps"] = measure_adjacent_steps(P, dev, local, peaks["hbm_gbs"])
         line["wavefront_rounds"] = measure_wavefront(P, dev, local, args.workload, K)
-        line["clip_at_once"] = measure_clip_at_once(P, dev, local)
+        line["peaked_logits"] = measure_peaked_logits(P, dev, local, args.workload, K)
+        line["clip_at_once"] = measure_clip_at_once(P, dev, local, group=27)
     if args.layers:
         line["profile_case"] = f"reduced to {args.layers} layers: not a benchmark result"
     if cpu_v is not None:
         line["cpu_baseline"] = dict(
             value=cpu_v, unit="TFLOP/s", cores=cpu_threads, kind="oracle", seconds=cpu_dt,
-            sample=(f"{CPU_SAMPLE_ROWS} of {w.chunk_frames * w.tokens_per_frame} query rows x {w.n_heads} heads of one "
-                    f"steady-state layer-call (N_kv={w.steady_n_kv()}), rotary+publish of the whole chunk included"),
+            sample=(f"{CPU_SAMPLE_ROWS or w.chunk_frames * w.tokens_per_frame} of {w.chunk_frames * w.tokens_per_frame} "
+                    f"query rows x {w.n_heads} heads of one steady-state layer-call (N_kv={w.steady_n_kv()}), rotary+publish "
+                    f"of the whole chunk included; a step of {w.n_stages * w.n_layers} such calls would take "
+                    f"{w.n_stages * w.n_layers}x as long (extrapolated, not timed)"),
             tiny_stream_in_full=oracle_tiny_stream())
     print(json.dumps(line), flush=True)
     if world > 1:

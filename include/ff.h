@@ -77,7 +77,7 @@ typedef struct {
                                     let several consecutive chunks of ONE stage share a batched launch, up to the
                                     full clip under the chunk-wise causal mask: n chunks need H + n slots.        */
     int32_t max_batch;           /* layer-calls per batched launch the arena has query regions for; 0 = min(S, 8);
-                                    at most FF_MAX_BATCH                                                         */
+                                    at most FF_MAX_BATCH (enough for every chunk of a 65 s clip in one launch)   */
     int32_t qk_norm;             /* nonzero: every (token, head) row of q and k is scaled by
                                     1/sqrt(mean(x^2) + qk_norm_eps) before the rotary embedding (the per-head
                                     normalisation that precedes this path in the backbone; fused into the same
@@ -180,7 +180,7 @@ ff_status ff_sched_run_node(ff_cache* c, int32_t stage, int32_t chunk_index, int
  * each stage its own device; on one device the same independence lets the nodes of a round share launches:
  * per layer, the rotations and publishes of all nodes, then ONE attention launch whose work list spans all of
  * them.  Results are identical, element for element, to issuing the calls one by one. */
-#define FF_MAX_BATCH 8
+#define FF_MAX_BATCH 128
 typedef struct {
     int32_t stage, chunk_index, n_frames, first_frame_pos;
     const void* q;   /* DEVICE, as in ff_chunk_forward_attn */
@@ -194,9 +194,14 @@ typedef struct {
  * checks of n_items ff_chunk_forward_attn calls issued in this order.  Items of different stages are independent.
  * Items of one stage must be consecutive chunks in order, starting at that stage's next chunk (the later ones
  * read what the earlier ones publish), and the bank must have H + (their number) slots (ring_slots): this is the
- * "full clip at once under a chunk-wise causal mask" form of Sec. 3, in groups of up to max_batch chunks.  All
- * items are checked before anything is enqueued or recorded: on an error status nothing has changed.
- * FF_ERR_UNSUPPORTED for more items than query regions or too few bank slots. */
+ * "full clip at once under a chunk-wise causal mask" form of Sec. 3: with ring_slots = H + N_R and max_batch = N_R
+ * every chunk of a stage shares ONE attention launch per layer.  Up to 8 items travel as launch arguments; beyond
+ * that the per-item descriptors are written to a page-locked host table (allocated by the library on first use:
+ * host memory, not device memory) and copied into the arena ahead of the attention launch on `stream`.  All
+ * items are checked before anything is enqueued, and the cache records the batch only after every launch has been
+ * accepted: on an error status - FF_ERR_CUDA included - the cache's tables and counters are as they were (kernels
+ * accepted before a failing launch may still run and write bank slots the tables do not list; such slots are
+ * never read).  FF_ERR_UNSUPPORTED for more items than query regions or too few bank slots. */
 ff_status ff_batch_forward_attn(ff_cache* c, int32_t layer, const ff_batch_item* items /*HOST*/, int32_t n_items,
                                 void* stream);
 typedef struct {
@@ -254,7 +259,14 @@ ff_status ff_cache_slot_ptr(const ff_cache* c, int32_t kind, int32_t stage, int3
                             void** k /*DEVICE out*/, void** v /*DEVICE out*/, int64_t strides[3],
                             int32_t* capacity_tokens);
 /* Synchronizes `stream` and returns the device status word (0 = no device-side error) in *word; the
- * function's own result is FF_ERR_TIMEOUT if a bounded wait expired.  Clears the word. */
+ * function's own result is FF_ERR_TIMEOUT if a bounded wait expired.  Clears the word.
+ * Every wait inside the kernels is bounded (2 s).  When one expires, the launch it belongs to records a code here,
+ * its other waits give up as well, and the kernel runs to its end without the data it waited for: the outputs and
+ * the bank slot of that layer-call are then UNDEFINED, and so is everything computed from them later.  The first
+ * code recorded stays until this function collects it; launches enqueued after the failing one run normally (an
+ * old code does not shorten their waits) but cannot record a second code.  Check the status at the points where
+ * results leave the stream (end of a chunk, of a clip), and treat everything since the previous check as lost
+ * when it is not FF_OK. */
 ff_status ff_cache_status(ff_cache* c, void* stream, uint32_t* word /*HOST out*/);
 /* Counters since creation/reset: layer-calls, Tail_H advances, anchor publishes, kernels launched. */
 ff_status ff_cache_counters(const ff_cache* c, int64_t* layer_calls, int64_t* advances, int64_t* anchor_publishes,
@@ -262,9 +274,10 @@ ff_status ff_cache_counters(const ff_cache* c, int64_t* layer_calls, int64_t* ad
 /* Per-kernel timing for roofline reports.  After ff_cache_profile_begin every layer-call records CUDA events
  * on its stream before the publish kernel, between the two kernels and after the attention kernel (at most
  * max_calls layer-calls are recorded; later ones run untimed; a batched call counts as one record, its publish
- * launch timed as one and its attention + merge launches as one).  ff_cache_profile_end synchronizes `stream`,
- * returns the summed kernel durations in milliseconds with the number of records behind each sum, and
- * releases the events.  Events are host-side driver objects; no device memory is allocated.  The events sit
+ * launches timed together and its attention + merge launches together).  ff_cache_profile_end synchronizes
+ * `stream`, returns the summed durations in milliseconds with the number of kernel launches behind each sum
+ * (publish_launches: publish kernels; attn_launches: attention kernels plus merge kernels), and releases the
+ * events.  Events are host-side driver objects; no device memory is allocated.  The events sit
  * between the kernels, so the overlap of a kernel's set-up with its predecessor's tail is not in these times. */
 ff_status ff_cache_profile_begin(ff_cache* c, int32_t max_calls);
 ff_status ff_cache_profile_end(ff_cache* c, void* stream, double* publish_ms, int64_t* publish_launches,
@@ -281,6 +294,11 @@ int32_t ff_debug_schedule(int32_t n_heads, int32_t n_items, const int32_t* n_q, 
  * for scores, 2 = scores ready, 3 = scores in registers, 4 = probabilities issued, 5 = probabilities stored;
  * issuer 10+ = waits for probabilities, 20+ = got them, 30+ = products issued (+2*tile + half). */
 ff_status ff_debug_set_trace(ff_cache* c, void* buf /*DEVICE*/, int32_t cap);
+/* Failure-injection hook, HOST only: the nth launch site from now (1 = the next publish / attention / merge
+ * launch of this cache; also counted on a bookkeeping-only cache) reports a failure without launching, so that
+ * the call it belongs to returns FF_ERR_CUDA.  Shows that a refused launch leaves the cache's tables untouched.
+ * nth = 0 disarms. */
+ff_status ff_debug_fail_launch(ff_cache* c, int32_t nth);
 /* Failure-detection hook: enqueues a one-thread kernel that waits limit_ns (<= 1e9) on a barrier nothing
  * will ever arrive on, gives up, and records an error in the status word, which the next ff_cache_status
  * reports as FF_ERR_TIMEOUT.  Shows that an expired device-side wait leaves the context usable. */
@@ -288,11 +306,14 @@ ff_status ff_debug_wait_probe(ff_cache* c, uint64_t limit_ns, void* stream);
 /* (No counterpart in the paper: an addition for callers that cannot allocate device memory.)
  * One layer-call on a FIRST chunk - empty history bank, no anchors - with no cache object and no arena:
  *   out = softmax(rope(q) rope(k)^T / sqrt(head_dim)) v   over the chunk's own n_frames*grid_h*grid_w tokens,
- * the same arithmetic as ff_chunk_forward_attn with chunk_index 0 and n_anchors 0 on the CUDA-core kernel.
+ * the same arithmetic as ff_chunk_forward_attn with chunk_index 0 and n_anchors 0 on the CUDA-core kernel (the
+ * rotary tables are evaluated by a small kernel on the device instead of on the host, so a table entry may
+ * differ from the arena path's in its last float bit).
  * Meant for code that receives device buffers but may not create any: a plug-in inside a process whose device
  * memory pool belongs to the host framework, a latency-critical loop that cannot afford cudaMalloc's implicit
  * synchronisation, or a process whose device memory was fully handed out before this library was loaded.
- * The call allocates nothing (no cudaMalloc, no cudaFree, no allocating library routine): its scratch - rotary
+ * The call allocates nothing (no cudaMalloc, no cudaFree, no allocating library routine, no host buffer) and
+ * copies nothing between host and device: it enqueues three kernels and returns.  Its scratch - rotary
  * tables, rotated queries, the rotated-K / V slot - is a fixed device array of FF_STATIC_SCRATCH_BYTES that
  * every GPU using this library holds until the process exits.
  *  - q, k, v, out: DEVICE, [n_frames*grid_h*grid_w, n_heads, head_dim], 16-byte aligned, dtype FF_BF16 or FF_F32;

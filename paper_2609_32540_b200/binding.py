@@ -26,7 +26,7 @@ SYMBOLS = [
     "ff_sched_run_chunk_host", "ff_sched_run_node", "ff_plan_anchor_count", "ff_plan_anchor_position",
     "ff_plan_window", "ff_cache_profile_begin", "ff_cache_profile_end",
     "ff_cache_ring_state", "ff_cache_anchor_state", "ff_cache_slot_ptr", "ff_cache_status",
-    "ff_cache_counters", "ff_debug_wait_probe", "ff_debug_set_trace", "ff_chunk_attn_static", "ff_cache_set_qk_gain",
+    "ff_cache_counters", "ff_debug_wait_probe", "ff_debug_fail_launch", "ff_debug_set_trace", "ff_chunk_attn_static", "ff_cache_set_qk_gain",
     "ff_euler_step", "ff_plan_sigma", "ff_batch_forward_attn", "ff_sched_run_round", "ff_debug_schedule", "ff_last_cuda_error", "ff_version",
 ]
 
@@ -67,7 +67,7 @@ class ff_round_node(C.Structure):
                 ("io", C.POINTER(ff_layer_io))]
 
 
-FF_MAX_BATCH = 8
+FF_MAX_BATCH = 128
 _lib = None
 
 
@@ -104,6 +104,7 @@ def load():
     L.ff_cache_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
     L.ff_cache_counters.argtypes = [vp, i64p, i64p, i64p, i64p]
     L.ff_debug_wait_probe.argtypes = [vp, C.c_uint64, vp]
+    L.ff_debug_fail_launch.argtypes = [vp, i32]
     L.ff_debug_set_trace.argtypes = [vp, vp, i32]
     L.ff_chunk_attn_static.argtypes = [i32, i32, i32, i32, i32, i32, C.c_float, i32, vp, vp, vp, vp, vp]
     L.ff_cache_set_qk_gain.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_float), vp]
@@ -294,6 +295,9 @@ class Cache:
 
     def ff_debug_set_trace(self, buf_ptr, cap) -> int:
         return load().ff_debug_set_trace(self._h, buf_ptr, cap)
+
+    def ff_debug_fail_launch(self, nth) -> int:
+        return load().ff_debug_fail_launch(self._h, nth)
 
     def ff_debug_wait_probe(self, limit_ns, stream=0) -> int:
         return load().ff_debug_wait_probe(self._h, limit_ns, stream)

@@ -23,8 +23,8 @@ template <>
 __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
 
 template <typename T, int D>
-__global__ void __launch_bounds__(256) attn_simt_kernel(const __grid_constant__ AttnArgs a, const int item_index) {
-    const AttnItem& item = a.items[item_index];
+__global__ void __launch_bounds__(256) attn_simt_kernel(const __grid_constant__ AttnArgs a) {
+    const AttnItem& item = a.items[0];
     constexpr int kRows = 64, kKeys = 32, kDpt = D / 4;
     __shared__ float sK[kKeys][D];
     __shared__ float sV[kKeys][D];
@@ -81,14 +81,19 @@ __global__ void __launch_bounds__(256) attn_simt_kernel(const __grid_constant__ 
     }
 }
 
-cudaError_t launch_attn_simt(const AttnArgs& a, int item, int dtype, cudaStream_t s) {
-    dim3 grid((a.items[item].n_q + 63) / 64, a.n_heads);
+// One launch per layer-call: `item` travels as the launch's only inline descriptor.
+cudaError_t launch_attn_simt(const AttnArgs& shared, const AttnItem& item, int dtype, cudaStream_t s) {
+    AttnArgs a = shared;
+    a.n_items = 1;
+    a.items_tab = nullptr;
+    a.items[0] = item;
+    dim3 grid((item.n_q + 63) / 64, a.n_heads);
     if (a.head_dim == 64) {
-        if (dtype == 0) attn_simt_kernel<__nv_bfloat16, 64><<<grid, 256, 0, s>>>(a, item);
-        else attn_simt_kernel<float, 64><<<grid, 256, 0, s>>>(a, item);
+        if (dtype == 0) attn_simt_kernel<__nv_bfloat16, 64><<<grid, 256, 0, s>>>(a);
+        else attn_simt_kernel<float, 64><<<grid, 256, 0, s>>>(a);
     } else if (a.head_dim == 128) {
-        if (dtype == 0) attn_simt_kernel<__nv_bfloat16, 128><<<grid, 256, 0, s>>>(a, item);
-        else attn_simt_kernel<float, 128><<<grid, 256, 0, s>>>(a, item);
+        if (dtype == 0) attn_simt_kernel<__nv_bfloat16, 128><<<grid, 256, 0, s>>>(a);
+        else attn_simt_kernel<float, 128><<<grid, 256, 0, s>>>(a);
     } else {
         return cudaErrorInvalidValue;
     }

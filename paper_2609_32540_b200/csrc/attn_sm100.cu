@@ -166,7 +166,7 @@ struct Tracer {
     }
 };
 
-template <int D, bool kTrace>
+template <int D, bool kTrace, bool kTable>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ AttnArgs a) {
@@ -221,24 +221,24 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             prefetch_tensormap(&tm_v);
             uint32_t kiter = 0, viter = 0, n_piece = 0;
             TileWalker w;
-            PieceIter pit;
+            PieceIter<kTable> pit;
             pit.init(a, cta);
             Piece p;
             for (; pit.next(a, p); ++n_piece) {
-                if (n_piece > 0) mbar_wait(&bar_q_empty, (n_piece - 1) & 1, a.status, kErrWaitQ);
+                if (n_piece > 0) mbar_wait(&bar_q_empty, (n_piece - 1) & 1, a.status, a.launch_tag | kErrWaitQ);
                 mbar_expect_tx(&bar_q_full, (p.two ? 2 : 1) * L::kTileBytes);
                 for (int t = 0; t < (p.two ? 2 : 1); ++t)
 #pragma unroll
                     for (int b = 0; b < D / 64; ++b)
                         tma_load_2d(smem + L::kQ + t * L::kTileBytes + b * L::kBoxBytes, &tm_q, b * 64,
-                                    a.items[p.item].q_row0 + p.h * a.q_rows_per_head + (2 * p.pr + t) * kTile,
+                                    item_at<kTable>(a, p.item).q_row0 + p.h * a.q_rows_per_head + (2 * p.pr + t) * kTile,
                                     &bar_q_full);
-                const KvSegs& segs = a.items[p.item].segs;
+                const KvSegs& segs = item_at<kTable>(a, p.item).segs;
                 w.seek(segs, p.j0);
                 for (int j = p.j0; j < p.j1; ++j) {
                     const int row = w.row(segs, p.h);
                     uint32_t st = kiter & 1;
-                    if (kiter >= 2) mbar_wait(&bar_k_empty[st], ((kiter >> 1) - 1) & 1, a.status, kErrWaitKEmpty);
+                    if (kiter >= 2) mbar_wait(&bar_k_empty[st], ((kiter >> 1) - 1) & 1, a.status, a.launch_tag | kErrWaitKEmpty);
                     mbar_expect_tx(&bar_k_full[st], L::kTileBytes);
 #pragma unroll
                     for (int b = 0; b < D / 64; ++b)
@@ -246,7 +246,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                                     &bar_k_full[st]);
                     ++kiter;
                     st = viter & 1;
-                    if (viter >= 2) mbar_wait(&bar_v_empty[st], ((viter >> 1) - 1) & 1, a.status, kErrWaitVEmpty);
+                    if (viter >= 2) mbar_wait(&bar_v_empty[st], ((viter >> 1) - 1) & 1, a.status, a.launch_tag | kErrWaitVEmpty);
                     mbar_expect_tx(&bar_v_full[st], L::kTileBytes);
 #pragma unroll
                     for (int b = 0; b < D / 64; ++b)
@@ -254,6 +254,16 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                                     &bar_v_full[st]);
                     ++viter;
                     w.next(segs);
+                }
+            }
+            // After an expired wait the roles stop consuming, so copies may still be on their way into shared
+            // memory: give the last ones a bounded time to land before the CTA ends and the memory is handed on.
+            if (*reinterpret_cast<volatile uint32_t*>(a.status) != 0u) {
+                constexpr unsigned long long kDrainNs = 5000000ull;
+                if (n_piece > 0) mbar_wait(&bar_q_full, (n_piece - 1) & 1, nullptr, 0, kDrainNs);
+                for (uint32_t back = 1; back <= 2; ++back) {
+                    if (kiter >= back) mbar_wait(&bar_k_full[(kiter - back) & 1], ((kiter - back) >> 1) & 1, nullptr, 0, kDrainNs);
+                    if (viter >= back) mbar_wait(&bar_v_full[(viter - back) & 1], ((viter - back) >> 1) & 1, nullptr, 0, kDrainNs);
                 }
             }
         }
@@ -279,14 +289,14 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             Tracer<kTrace> tr;
             tr.init(a, 2, cta == 0 && t == 0 && leader != 0);
 
-            PieceIter pit;
+            PieceIter<kTable> pit;
             pit.init(a, cta);
             Piece p;
             for (; pit.next(a, p); ++n_piece) {
                 const bool active = (t == 0) || p.two;  // an idle stream still takes part in the K/V/Q hand-back
-                mbar_wait(&bar_q_full, n_piece & 1, a.status, kErrWaitQ);
+                mbar_wait(&bar_q_full, n_piece & 1, a.status, a.launch_tag | kErrWaitQ);
                 uint32_t k_cur = k_lo0 + (kiter & 1) * (L::kTileBytes >> 4);
-                mbar_wait(&bar_k_full[kiter & 1], (kiter >> 1) & 1, a.status, kErrWaitK);
+                mbar_wait(&bar_k_full[kiter & 1], (kiter >> 1) & 1, a.status, a.launch_tag | kErrWaitK);
                 tc_fence_after_sync();
                 if (active) {
 #pragma unroll
@@ -301,8 +311,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 // The V tile of a key tile and the K tile of the next one are waited for one key tile ahead, while
                 // this thread would otherwise just wait for the first probabilities: a barrier wait costs it
                 // more than a hundred cycles even when the barrier is ready, and that would delay the products.
-                mbar_wait(&bar_v_full[viter & 1], (viter >> 1) & 1, a.status, kErrWaitV);
-                if (p.j1 - p.j0 > 1) mbar_wait(&bar_k_full[kiter & 1], (kiter >> 1) & 1, a.status, kErrWaitK);
+                mbar_wait(&bar_v_full[viter & 1], (viter >> 1) & 1, a.status, a.launch_tag | kErrWaitV);
+                if (p.j1 - p.j0 > 1) mbar_wait(&bar_k_full[kiter & 1], (kiter >> 1) & 1, a.status, a.launch_tag | kErrWaitK);
                 for (int j = p.j0; j < p.j1; ++j) {
                     const bool last = (j == p.j1 - 1);
                     const uint32_t vst = viter & 1, kst = kiter & 1;
@@ -312,7 +322,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                         for (int b = 0; b < kNB; ++b) {
                             tr.mark(10 + b);
-                            mbar_wait(&bar_p_full[t][b], sp & 1, a.status, kErrWaitP);
+                            mbar_wait(&bar_p_full[t][b], sp & 1, a.status, a.launch_tag | kErrWaitP);
                             tr.mark(20 + b);
                             tc_fence_after_sync();
                             // O_t += P_t[b] . V(keys 64b..64b+63): 16 keys per product = two groups of 8 rows of
@@ -339,8 +349,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         // the scores of the piece's last key tile have just been issued: Q is no longer needed and
                         // the producer may fetch the next piece's query tiles while this piece finishes
                         if (j + 2 == p.j1) mma_commit_p(&bar_q_empty, leader);
-                        mbar_wait(&bar_v_full[viter & 1], (viter >> 1) & 1, a.status, kErrWaitV);
-                        if (j + 2 < p.j1) mbar_wait(&bar_k_full[kiter & 1], (kiter >> 1) & 1, a.status, kErrWaitK);
+                        mbar_wait(&bar_v_full[viter & 1], (viter >> 1) & 1, a.status, a.launch_tag | kErrWaitV);
+                        if (j + 2 < p.j1) mbar_wait(&bar_k_full[kiter & 1], (kiter >> 1) & 1, a.status, a.launch_tag | kErrWaitK);
                     }
                 }
             }
@@ -357,14 +367,14 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         Tracer<kTrace> tr;
         tr.init(a, t, cta == 0 && r == 0);
         TileWalker w;
-        PieceIter pit;
+        PieceIter<kTable> pit;
         pit.init(a, cta);
         Piece p;
         while (pit.next(a, p)) {
             if (t == 1 && !p.two) continue;
             float m_used = -INFINITY;  // raw-score maximum the exponents are taken against
             float l = 0.f;
-            const AttnItem& item = a.items[p.item];
+            const AttnItem& item = item_at<kTable>(a, p.item);
             w.seek(item.segs, p.j0);
             for (int j = p.j0; j < p.j1; ++j, ++sp) {
                 const int n_valid = w.n_valid(item.segs);
@@ -373,7 +383,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int b = 0; b < kNB; ++b, ++halves) {
                     const int n_here = n_valid - b * kHalf;  // valid key columns of this half (may be <= 0)
                     tr.mark(1);
-                    mbar_wait(&bar_s_full[t][b], sp & 1, a.status, kErrWaitS);
+                    mbar_wait(&bar_s_full[t][b], sp & 1, a.status, a.launch_tag | kErrWaitS);
                     tr.mark(2);
                     tc_fence_after_sync();
                     uint32_t sr[kHalf / 32][32];
@@ -403,7 +413,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         const float m_new = fmaxf(m_used, tmax);
                         if (j > p.j0 || b > 0) {
                             // O_t may only be touched once the product fed by the previous half tile has finished
-                            mbar_wait(&bar_pv_done[t], (halves - 1) & 1, a.status, kErrWaitO);
+                            mbar_wait(&bar_pv_done[t], (halves - 1) & 1, a.status, a.launch_tag | kErrWaitO);
                             tc_fence_after_sync();
                             const float alpha = ex2_approx((m_used - m_new) * c);
                             l *= alpha;
@@ -452,7 +462,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
             }
             // epilogue of the piece
-            mbar_wait(&bar_o_full[t], op & 1, a.status, kErrWaitO);
+            mbar_wait(&bar_o_full[t], op & 1, a.status, a.launch_tag | kErrWaitO);
             ++op;
             tc_fence_after_sync();
             const int row = (2 * p.pr + t) * kTile + r;
@@ -505,7 +515,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 // out = sum_i 2^(m_i - m*) O_i / sum_i 2^(m_i - m*) l_i.  One warp per query row (a lane owns D/32 columns),
 // 8 rows per block, so that enough rows are in flight to hide the latency of the scattered reads.  The grid
 // covers the remainder pairs only (whole pairs store their final result themselves).
-template <int D>
+template <int D, bool kTable>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const __grid_constant__ AttnArgs a) {
     constexpr int kPerLane = D / 32;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -516,8 +526,8 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const __grid_constant
     const int rr = static_cast<int>(gr % (2 * kTile));
     const long long cz = a.iters_per_cta;
     int it_i;
-    const long long s_g = rem_iter_start(a, g, &it_i);
-    const AttnItem& item = a.items[it_i];
+    const long long s_g = rem_iter_start<kTable>(a, g, &it_i);
+    const AttnItem& item = item_at<kTable>(a, it_i);
     const long long e_g = s_g + item.n_kv_tiles;
     const int first = static_cast<int>(s_g / cz);
     const int last = static_cast<int>((e_g - 1) / cz);
@@ -564,11 +574,13 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const __grid_constant
 
 template <int D>
 static cudaError_t set_smem() {
-    cudaError_t e = cudaFuncSetAttribute(attn_tcgen05_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         SmemLayout<D>::kDynamic);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(attn_tcgen05_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                SmemLayout<D>::kDynamic);
+    const int bytes = SmemLayout<D>::kDynamic;
+    cudaError_t e = cudaFuncSetAttribute(attn_tcgen05_kernel<D, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(attn_tcgen05_kernel<D, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(attn_tcgen05_kernel<D, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    return e;
 }
 
 cudaError_t attn_tcgen05_prepare(int head_dim) {
@@ -579,12 +591,14 @@ cudaError_t attn_tcgen05_prepare(int head_dim) {
     return cudaErrorInvalidValue;
 }
 
-// Fills the schedule fields of `a` for at most `n_ctas_max` resident CTAs; returns the number of remainder pairs
-// if some of them are cut (their pieces need merging), else 0.
-int attn_tcgen05_plan(AttnArgs& a, int n_ctas_max) {
+// Fills the schedule fields of `a` and of its n_items descriptors `items` (host memory: the array inside `a`, or
+// the host copy of the table) for at most `n_ctas_max` resident CTAs; returns the number of remainder pairs if
+// some of them are cut (their pieces need merging), else 0.
+template <bool kTable>
+static int plan_impl(AttnArgs& a, AttnItem* items, int n_ctas_max) {
     long long n_pairs = 0, work = 0;
     for (int i = 0; i < a.n_items; ++i) {
-        AttnItem& I = a.items[i];
+        AttnItem& I = items[i];
         I.n_qt = (I.n_q + kTile - 1) / kTile;
         I.n_qp = (I.n_qt + 1) / 2;
         int tiles = 0;
@@ -603,7 +617,7 @@ int attn_tcgen05_plan(AttnArgs& a, int n_ctas_max) {
     const long long g0 = static_cast<long long>(a.n_full) * n_cta;  // first pair shared out by key-tile ranges
     long long iters = 0;
     for (int i = 0; i < a.n_items; ++i) {
-        AttnItem& I = a.items[i];
+        AttnItem& I = items[i];
         const long long pairs = static_cast<long long>(a.n_heads) * I.n_qp;
         long long first_rem = g0 - I.pair0;
         if (first_rem < 0) first_rem = 0;
@@ -617,31 +631,46 @@ int attn_tcgen05_plan(AttnArgs& a, int n_ctas_max) {
     bool cut = false;
     for (long long g = g0; g < n_pairs && !cut; ++g) {
         int it_i;
-        const long long s_g = rem_iter_start(a, static_cast<int>(g), &it_i);
-        cut = s_g / a.iters_per_cta != (s_g + a.items[it_i].n_kv_tiles - 1) / a.iters_per_cta;
+        const long long s_g = rem_iter_start<kTable>(a, static_cast<int>(g), &it_i);
+        cut = s_g / a.iters_per_cta != (s_g + items[it_i].n_kv_tiles - 1) / a.iters_per_cta;
     }
     return cut ? static_cast<int>(n_pairs - g0) : 0;
 }
 
-cudaError_t launch_attn_tcgen05(AttnArgs& a, int n_ctas_max, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
-                                const CUtensorMap& tm_v, cudaStream_t s, int* n_launches) {
-    const int merge_pairs = attn_tcgen05_plan(a, n_ctas_max);
-    *n_launches = merge_pairs ? 2 : 1;
-    const bool trace = a.trace != nullptr;
-    const dim3 grid(a.n_ctas), block(kThreads), mgrid(merge_pairs * (2 * kTile / 8)), mblock(256);
-    cudaError_t e;
-    if (a.head_dim == 128) {
-        e = trace ? launch_overlapped(attn_tcgen05_kernel<128, true>, grid, block, SmemLayout<128>::kDynamic, s, tm_q, tm_k, tm_v, a)
-                  : launch_overlapped(attn_tcgen05_kernel<128, false>, grid, block, SmemLayout<128>::kDynamic, s, tm_q, tm_k, tm_v, a);
-        if (e == cudaSuccess && merge_pairs) e = launch_overlapped(attn_combine_kernel<128>, mgrid, mblock, 0, s, a);
-    } else if (a.head_dim == 64) {
-        e = trace ? launch_overlapped(attn_tcgen05_kernel<64, true>, grid, block, SmemLayout<64>::kDynamic, s, tm_q, tm_k, tm_v, a)
-                  : launch_overlapped(attn_tcgen05_kernel<64, false>, grid, block, SmemLayout<64>::kDynamic, s, tm_q, tm_k, tm_v, a);
-        if (e == cudaSuccess && merge_pairs) e = launch_overlapped(attn_combine_kernel<64>, mgrid, mblock, 0, s, a);
-    } else {
-        return cudaErrorInvalidValue;
+int attn_tcgen05_plan(AttnArgs& a, AttnItem* items, int n_ctas_max) {
+    if (items == a.items) {
+        a.items_tab = nullptr;
+        return plan_impl<false>(a, items, n_ctas_max);
     }
+    a.items_tab = items;
+    return plan_impl<true>(a, items, n_ctas_max);
+}
+
+// `a` has been planned (attn_tcgen05_plan returned merge_pairs); with more than kMaxInline items a.items_tab must
+// point to the device copy of the planned descriptors.
+template <int D>
+static cudaError_t launch_impl(const AttnArgs& a, int merge_pairs, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
+                               const CUtensorMap& tm_v, cudaStream_t s) {
+    const bool table = a.items_tab != nullptr, trace = a.trace != nullptr && !table;
+    const dim3 grid(a.n_ctas), block(kThreads), mgrid(merge_pairs * (2 * kTile / 8)), mblock(256);
+    const size_t smem = SmemLayout<D>::kDynamic;
+    cudaError_t e;
+    if (table) e = launch_overlapped(attn_tcgen05_kernel<D, false, true>, grid, block, smem, s, tm_q, tm_k, tm_v, a);
+    else if (trace) e = launch_overlapped(attn_tcgen05_kernel<D, true, false>, grid, block, smem, s, tm_q, tm_k, tm_v, a);
+    else e = launch_overlapped(attn_tcgen05_kernel<D, false, false>, grid, block, smem, s, tm_q, tm_k, tm_v, a);
+    if (e == cudaSuccess && merge_pairs)
+        e = table ? launch_overlapped(attn_combine_kernel<D, true>, mgrid, mblock, 0, s, a)
+                  : launch_overlapped(attn_combine_kernel<D, false>, mgrid, mblock, 0, s, a);
     return e;
+}
+
+cudaError_t launch_attn_tcgen05(const AttnArgs& a, int merge_pairs, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
+                                const CUtensorMap& tm_v, cudaStream_t s, int* n_launches) {
+    *n_launches = merge_pairs ? 2 : 1;
+    if (a.n_items > kMaxInline && !a.items_tab) return cudaErrorInvalidValue;
+    if (a.head_dim == 128) return launch_impl<128>(a, merge_pairs, tm_q, tm_k, tm_v, s);
+    if (a.head_dim == 64) return launch_impl<64>(a, merge_pairs, tm_q, tm_k, tm_v, s);
+    return cudaErrorInvalidValue;
 }
 
 // A one-thread kernel that waits on a barrier nothing arrives on, with a short limit: exercises the bounded

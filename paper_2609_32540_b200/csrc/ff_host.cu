@@ -34,7 +34,7 @@ struct Derived {
     int32_t tf, cap, cap_pad, tf_pad, elem, d, pairs[3], q_slots;
     int32_t R;  // slots per bank: H + 1 unless the caller asked for more (several chunks of one stage per launch)
     int64_t ring_rows, anchor_rows, total_rows;
-    size_t off_tab_f, off_tab_y, off_tab_x, off_status, off_gain, off_k, off_v, off_q, off_part_o, off_part_ml, off_stage, stage_bytes, total;
+    size_t off_tab_f, off_tab_y, off_tab_x, off_status, off_items, off_gain, off_k, off_v, off_q, off_part_o, off_part_ml, off_stage, stage_bytes, total;
     int impl;
 };
 
@@ -53,6 +53,7 @@ ff_status derive(const ff_cache_config* cfg, Derived* D) {
     if (cfg->max_batch < 0 || cfg->max_batch > kMaxBatch) return FF_ERR_INVALID_ARG;
     D->R = cfg->ring_slots ? cfg->ring_slots : cfg->history_chunks + 1;
     if (cfg->max_visible_anchors > cfg->n_anchor_slots) return FF_ERR_INVALID_ARG;
+    static_assert(FF_MAX_BATCH == kMaxBatch, "ff.h and ff_internal.h disagree on the batch limit");
     if (cfg->head_dim != 64 && cfg->head_dim != 128) return FF_ERR_UNSUPPORTED;
     int impl = cfg->attn_impl;
     if (impl == FF_ATTN_AUTO) impl = cfg->dtype == FF_BF16 ? FF_ATTN_TCGEN05 : FF_ATTN_SIMT;
@@ -89,13 +90,15 @@ ff_status derive(const ff_cache_config* cfg, Derived* D) {
     D->off_tab_y = off; off = align_up(off + (size_t)cfg->grid_h * D->pairs[1] * sizeof(float2), 256);
     D->off_tab_x = off; off = align_up(off + (size_t)cfg->grid_w * D->pairs[2] * sizeof(float2), 256);
     D->off_status = off; off = align_up(off + 256, 1024);
+    // descriptors of a launch over more than kMaxInline layer-calls (the whole clip of a stage at once)
+    D->off_items = off; off = align_up(off + (size_t)kMaxBatch * sizeof(AttnItem), 1024);
     // channel gains of the q/k normalisation: [layer][q|k][d] floats; absent when the normalisation is off
     D->off_gain = off; off = align_up(off + (cfg->qk_norm ? (size_t)cfg->n_layers * 2 * D->d * sizeof(float) : 0), 1024);
     const size_t mat_bytes = (size_t)D->total_rows * D->d * D->elem;
     D->off_k = off; off = align_up(off + mat_bytes, 1024);
     D->off_v = off; off = align_up(off + mat_bytes, 1024);
     // rotated queries: one region per layer-call of a batched launch (at most one call per stage)
-    D->q_slots = cfg->max_batch ? cfg->max_batch : (cfg->n_stages < kMaxBatch ? cfg->n_stages : kMaxBatch);
+    D->q_slots = cfg->max_batch ? cfg->max_batch : (cfg->n_stages < kMaxInline ? cfg->n_stages : kMaxInline);
     D->off_q = off; off = align_up(off + (size_t)D->q_slots * cfg->n_heads * D->cap_pad * D->d * D->elem, 1024);
     D->off_part_o = off; off = align_up(off + (size_t)2 * kMaxCtas * 2 * kTile * D->d * sizeof(float), 1024);
     D->off_part_ml = off; off = align_up(off + (size_t)2 * kMaxCtas * 2 * kTile * sizeof(float2), 1024);
@@ -133,6 +136,14 @@ struct ff_cache {
                 ev_out[2] = {nullptr, nullptr};
     unsigned long long* trace = nullptr;  // device buffer for the attention kernel's event trace (caller-owned)
     int32_t trace_cap = 0;
+    // page-locked host copies of the descriptor table of launches over more than kMaxInline layer-calls; two, used
+    // in turn, each guarded by an event that says its upload has finished (created on first use)
+    AttnItem* host_tab[2] = {nullptr, nullptr};
+    cudaEvent_t tab_ev[2] = {nullptr, nullptr};
+    int tab_turn = 0;
+    uint32_t launch_seq = 0;        // numbers the attention launches; tags the error codes a launch records
+    int32_t fail_launch_in = 0;     // test hook: the n-th launch site from now reports a failure without launching
+    int64_t prof_publish_launches = 0, prof_attn_launches = 0;
 
     SlotMeta& slot(int stage, int layer, int s) {
         return slots[((size_t)stage * cfg.n_layers + layer) * D.R + s];
@@ -161,6 +172,14 @@ struct ff_cache {
         return reinterpret_cast<const float*>(arena + D.off_gain) + ((size_t)layer * 2 + which) * D.d;
     }
     uint32_t* status() const { return reinterpret_cast<uint32_t*>(arena + D.off_status); }
+    // A launch site: true if the launch may proceed; false when the test hook turns it into a reported failure.
+    bool launch_allowed() {
+        if (fail_launch_in > 0 && --fail_launch_in == 0) {
+            g_last_cuda_error = static_cast<int32_t>(cudaErrorLaunchFailure);
+            return false;
+        }
+        return true;
+    }
 };
 
 namespace {
@@ -324,6 +343,8 @@ ff_status ff_cache_destroy(ff_cache* c) {
         if (c->s_out) cudaStreamDestroy(c->s_out);
         if (c->ev_entry) cudaEventDestroy(c->ev_entry);
         for (int i = 0; i < 2; ++i) {
+            if (c->host_tab[i]) cudaFreeHost(c->host_tab[i]);
+            if (c->tab_ev[i]) cudaEventDestroy(c->tab_ev[i]);
             if (c->ev_in[i]) cudaEventDestroy(c->ev_in[i]);
             if (c->ev_done[i]) cudaEventDestroy(c->ev_done[i]);
             if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
@@ -346,6 +367,7 @@ ff_status ff_cache_profile_begin(ff_cache* c, int32_t max_calls) {
         }
     }
     c->prof_used = 0;
+    c->prof_publish_launches = c->prof_attn_launches = 0;
     c->profiling = true;
     return FF_OK;
 }
@@ -358,7 +380,6 @@ ff_status ff_cache_profile_end(ff_cache* c, void* stream, double* publish_ms, in
     ff_status r = FF_OK;
     if (!cuda_ok(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)))) r = FF_ERR_CUDA;
     double pm = 0.0, am = 0.0;
-    int64_t n = 0;
     for (size_t i = 0; r == FF_OK && i + 3 <= c->prof_used; i += 3) {
         float a = 0.f, b = 0.f;
         if (!cuda_ok(cudaEventElapsedTime(&a, c->prof_events[i], c->prof_events[i + 1])) ||
@@ -368,15 +389,14 @@ ff_status ff_cache_profile_end(ff_cache* c, void* stream, double* publish_ms, in
         }
         pm += a;
         am += b;
-        ++n;
     }
     for (cudaEvent_t e : c->prof_events) cudaEventDestroy(e);
     c->prof_events.clear();
     c->prof_used = 0;
     if (publish_ms) *publish_ms = pm;
     if (attn_ms) *attn_ms = am;
-    if (publish_launches) *publish_launches = n;
-    if (attn_launches) *attn_launches = n;
+    if (publish_launches) *publish_launches = c->prof_publish_launches;
+    if (attn_launches) *attn_launches = c->prof_attn_launches;
     return r;
 }
 
@@ -417,6 +437,7 @@ ff_status ff_anchor_publish(ff_cache* c, int32_t slot, int32_t frame_pos, int32_
     a.qk_norm = c->cfg.qk_norm; a.qk_norm_eps = c->cfg.qk_norm_eps;
     a.gain_q = c->gain(layer, 0); a.gain_k = c->gain(layer, 1);
     a.tab = c->tables();
+    if (!c->launch_allowed()) return FF_ERR_CUDA;
     if (!c->dry) {
         if (!cuda_ok(launch_rope_publish(a, c->cfg.dtype, c->sm_count, static_cast<cudaStream_t>(stream))))
             return FF_ERR_CUDA;
@@ -479,9 +500,11 @@ ff_status validate_call(const ff_cache* c, int32_t layer, const CallDesc& d, int
 // must be consecutive chunks in order - a later chunk reads what the earlier ones publish in the same batch,
 // which is complete before the attention launch starts - and the bank needs H + (their number) slots so that no
 // publish overwrites a chunk an earlier call still reads.
+// Nothing of the cache's state (slot table, counters, profile records) is touched before every launch of the
+// batch has been accepted by the runtime: on any error status the cache is as it was.
 ff_status forward_batch(ff_cache* c, int32_t layer, const CallDesc* d, int32_t n, cudaStream_t s) {
     if (!c || !d || n < 1) return FF_ERR_INVALID_ARG;
-    if (n > c->D.q_slots) return FF_ERR_UNSUPPORTED;
+    if (n > c->D.q_slots || n > kMaxBatch) return FF_ERR_UNSUPPORTED;
     const ff_cache_config& cfg = c->cfg;
     for (int i = 0; i < n; ++i) {
         int pos = 0;
@@ -491,25 +514,53 @@ ff_status forward_batch(ff_cache* c, int32_t layer, const CallDesc* d, int32_t n
         if (r != FF_OK) return r;
     }
     const int H = cfg.history_chunks, R = c->D.R;
+    const bool table = n > kMaxInline;
     cudaEvent_t* ev = nullptr;
-    if (c->profiling && c->prof_used + 3 <= c->prof_events.size()) {
-        ev = &c->prof_events[c->prof_used];
-        c->prof_used += 3;
-    }
+    if (!c->dry && c->profiling && c->prof_used + 3 <= c->prof_events.size()) ev = &c->prof_events[c->prof_used];
+
     AttnArgs a{};
     a.q_rot = c->arena + c->D.off_q; a.kmat = c->arena + c->D.off_k; a.vmat = c->arena + c->D.off_v;
     a.q_rows_per_head = c->D.cap_pad;
     a.n_heads = cfg.n_heads; a.head_dim = c->D.d;
     a.scale = 1.0f / std::sqrt((float)c->D.d);
     a.status = c->status();
+    a.launch_tag = ((c->launch_seq + 1) & 0x7fffu) << 16;
     a.n_items = n;
     a.part_o = reinterpret_cast<float*>(c->arena + c->D.off_part_o);
     a.part_ml = reinterpret_cast<float2*>(c->arena + c->D.off_part_ml);
     a.trace = c->trace;
     a.trace_cap = c->trace_cap;
-    if (!c->dry && ev) cudaEventRecord(ev[0], s);
-    PublishBatch pb{};
-    pb.n = n;
+
+    // where the descriptors are written: inside the launch arguments, or (many calls) a page-locked host table that
+    // is copied into the arena ahead of the attention launch
+    std::vector<AttnItem> dry_items;
+    AttnItem* items = a.items;
+    const int turn = c->tab_turn;
+    if (table) {
+        if (c->dry) {
+            dry_items.resize(n);
+            items = dry_items.data();
+        } else {
+            for (int b = 0; b < 2; ++b) {
+                if (!c->host_tab[b] &&
+                    (!cuda_ok(cudaHostAlloc(reinterpret_cast<void**>(&c->host_tab[b]), kMaxBatch * sizeof(AttnItem), cudaHostAllocDefault)) ||
+                     !cuda_ok(cudaEventCreateWithFlags(&c->tab_ev[b], cudaEventDisableTiming))))
+                    return FF_ERR_CUDA;
+            }
+            if (!cuda_ok(cudaEventSynchronize(c->tab_ev[turn]))) return FF_ERR_CUDA;  // its previous upload is done
+            items = c->host_tab[turn];
+        }
+    }
+
+    // slots this batch publishes: visible to its later calls, recorded in the cache only at the end
+    struct Pending { int32_t stage, slot, chunk, n_tokens; };
+    Pending pend[kMaxBatch];
+    auto tokens_in = [&](int upto, int stage, int sl) -> int32_t {
+        for (int j = upto; j >= 0; --j)
+            if (pend[j].stage == stage && pend[j].slot == sl) return pend[j].n_tokens;
+        return c->slot(stage, layer, sl).n_tokens;
+    };
+    std::vector<PublishArgs> pubs(n);
     for (int i = 0; i < n; ++i) {
         const CallDesc& x = d[i];
         const int n_q = x.n_frames * c->D.tf;
@@ -517,7 +568,8 @@ ff_status forward_batch(ff_cache* c, int32_t layer, const CallDesc* d, int32_t n
         const int64_t q_row0 = (int64_t)i * cfg.n_heads * c->D.cap_pad;
 
         // steps 1-2: rotate Q and K, publish (K', V) in place into the stage's ring slot
-        PublishArgs& p = pb.items[i];
+        PublishArgs& p = pubs[i];
+        p = PublishArgs{};
         p.q = x.q; p.k = x.k; p.v = x.v;
         p.q_rot = c->arena + c->D.off_q + (size_t)q_row0 * c->D.d * c->D.elem;
         p.kmat = c->arena + c->D.off_k; p.vmat = c->arena + c->D.off_v;
@@ -531,11 +583,11 @@ ff_status forward_batch(ff_cache* c, int32_t layer, const CallDesc* d, int32_t n
         p.qk_norm = cfg.qk_norm; p.qk_norm_eps = cfg.qk_norm_eps;
         p.gain_q = c->gain(layer, 0); p.gain_k = c->gain(layer, 1);
         p.tab = c->tables();
-        c->slot(x.stage, layer, own).chunk = x.chunk_index;
-        c->slot(x.stage, layer, own).n_tokens = n_q;
+        pend[i] = Pending{x.stage, own, x.chunk_index, n_q};
 
         // steps 3-4: attention over [anchors | history | own], read where they lie
-        AttnItem& it = a.items[i];
+        AttnItem& it = items[i];
+        it = AttnItem{};
         it.out = x.out;
         it.q_row0 = (int32_t)q_row0;
         it.n_q = n_q;
@@ -550,29 +602,65 @@ ff_status forward_batch(ff_cache* c, int32_t layer, const CallDesc* d, int32_t n
             const int sl = j % R;
             it.segs.row0[m] = (int32_t)c->ring_row0(x.stage, layer, sl);
             it.segs.head_stride[m] = c->ring_head_stride();
-            it.segs.tokens[m] = c->slot(x.stage, layer, sl).n_tokens;
+            it.segs.tokens[m] = tokens_in(i, x.stage, sl);
         }
         it.segs.n = m;
     }
-    if (!c->dry) {
-        // one launch publishes every item (the items write disjoint slots and query regions)
-        if (!cuda_ok(launch_rope_publish_batch(pb, cfg.dtype, c->sm_count, s))) return FF_ERR_CUDA;
-        ++c->n_launches;
-        if (ev) cudaEventRecord(ev[1], s);
-        if (c->D.impl == FF_ATTN_TCGEN05) {
-            int launched = 1;
-            if (!cuda_ok(launch_attn_tcgen05(a, c->sm_count < kMaxCtas ? c->sm_count : kMaxCtas, c->tm_q, c->tm_k, c->tm_v,
-                                             s, &launched)))
-                return FF_ERR_CUDA;
-            c->n_launches += launched;
-        } else {
-            for (int i = 0; i < n; ++i) {
-                if (!cuda_ok(launch_attn_simt(a, i, cfg.dtype, s))) return FF_ERR_CUDA;
-                ++c->n_launches;
-            }
-        }
-        if (ev) cudaEventRecord(ev[2], s);
+    const bool tc = c->D.impl == FF_ATTN_TCGEN05;
+    const int merge_pairs = tc ? attn_tcgen05_plan(a, items, c->sm_count < kMaxCtas ? c->sm_count : kMaxCtas) : 0;
+
+    int64_t launched = 0, pub_launches = 0, attn_launches = 0;
+    if (ev) cudaEventRecord(ev[0], s);
+    // the publishes, kMaxInline per launch (the items write disjoint slots and query regions)
+    for (int i0 = 0; i0 < n; i0 += kMaxInline) {
+        PublishBatch pb{};
+        pb.n = n - i0 < kMaxInline ? n - i0 : kMaxInline;
+        for (int i = 0; i < pb.n; ++i) pb.items[i] = pubs[i0 + i];
+        if (!c->launch_allowed()) return FF_ERR_CUDA;
+        if (!c->dry && !cuda_ok(launch_rope_publish_batch(pb, cfg.dtype, c->sm_count, s))) return FF_ERR_CUDA;
+        ++pub_launches;
     }
+    if (ev) cudaEventRecord(ev[1], s);
+    if (tc) {
+        if (!c->launch_allowed()) return FF_ERR_CUDA;
+        if (!c->dry) {
+            if (table) {
+                AttnItem* dev_tab = reinterpret_cast<AttnItem*>(c->arena + c->D.off_items);
+                if (!cuda_ok(cudaMemcpyAsync(dev_tab, items, (size_t)n * sizeof(AttnItem), cudaMemcpyHostToDevice, s)) ||
+                    !cuda_ok(cudaEventRecord(c->tab_ev[turn], s)))
+                    return FF_ERR_CUDA;
+                c->tab_turn ^= 1;
+                a.items_tab = dev_tab;
+            }
+            int nl = 1;
+            if (!cuda_ok(launch_attn_tcgen05(a, merge_pairs, c->tm_q, c->tm_k, c->tm_v, s, &nl))) return FF_ERR_CUDA;
+            attn_launches += nl;
+        } else {
+            attn_launches += merge_pairs ? 2 : 1;
+        }
+    } else {
+        for (int i = 0; i < n; ++i) {
+            if (!c->launch_allowed()) return FF_ERR_CUDA;
+            if (!c->dry && !cuda_ok(launch_attn_simt(a, items[i], cfg.dtype, s))) return FF_ERR_CUDA;
+            ++attn_launches;
+        }
+    }
+    if (ev) cudaEventRecord(ev[2], s);
+    launched = pub_launches + attn_launches;
+
+    // every launch was accepted: now the cache records what they do
+    for (int i = 0; i < n; ++i) {
+        SlotMeta& m = c->slot(pend[i].stage, layer, pend[i].slot);
+        m.chunk = pend[i].chunk;
+        m.n_tokens = pend[i].n_tokens;
+    }
+    ++c->launch_seq;
+    if (ev) {
+        c->prof_used += 3;
+        c->prof_publish_launches += pub_launches;
+        c->prof_attn_launches += attn_launches;
+    }
+    if (!c->dry) c->n_launches += launched;
     c->n_layer_calls += n;
     return FF_OK;
 }
@@ -800,7 +888,7 @@ ff_status ff_cache_status(ff_cache* c, void* stream, uint32_t* word) {
     if (!cuda_ok(cudaStreamSynchronize(s))) return FF_ERR_CUDA;
     if (!cuda_ok(cudaMemcpy(&w, c->status(), sizeof(w), cudaMemcpyDeviceToHost))) return FF_ERR_CUDA;
     if (w != 0 && !cuda_ok(cudaMemset(c->status(), 0, sizeof(w)))) return FF_ERR_CUDA;
-    if (word) *word = w;
+    if (word) *word = w & 0xffffu;  // the upper half says which launch recorded it
     return w == 0 ? FF_OK : FF_ERR_TIMEOUT;
 }
 
@@ -827,27 +915,32 @@ int32_t ff_debug_schedule(int32_t n_heads, int32_t n_items, const int32_t* n_q, 
     AttnArgs a{};
     a.n_heads = n_heads;
     a.n_items = n_items;
+    std::vector<AttnItem> tab(n_items > kMaxInline ? n_items : 0);
+    AttnItem* items = n_items > kMaxInline ? tab.data() : a.items;
     for (int i = 0; i < n_items; ++i) {
         if (n_q[i] < 1 || n_kv[i] < 1) return -1;
-        a.items[i].n_q = n_q[i];
-        a.items[i].segs.n = 1;
-        a.items[i].segs.tokens[0] = n_kv[i];
+        items[i] = AttnItem{};
+        items[i].n_q = n_q[i];
+        items[i].segs.n = 1;
+        items[i].segs.tokens[0] = n_kv[i];
     }
-    const int merge_pairs = attn_tcgen05_plan(a, n_ctas_max);
+    const int merge_pairs = attn_tcgen05_plan(a, items, n_ctas_max);
     if (header) { header[0] = a.n_ctas; header[1] = a.n_full; header[2] = merge_pairs; header[3] = a.iters_per_cta; }
     int32_t n = 0;
-    for (int cta = 0; cta < a.n_ctas; ++cta) {
-        PieceIter pit;
-        pit.init(a, cta);
-        Piece p;
-        while (pit.next(a, p)) {
-            if (n < cap) {
-                int32_t* r = records + (size_t)n * 8;
-                r[0] = cta; r[1] = p.item; r[2] = p.h; r[3] = p.pr; r[4] = p.j0; r[5] = p.j1; r[6] = p.slot; r[7] = p.two;
+    auto walk = [&](auto pit) {
+        for (int cta = 0; cta < a.n_ctas; ++cta) {
+            pit.init(a, cta);
+            Piece p;
+            while (pit.next(a, p)) {
+                if (n < cap) {
+                    int32_t* r = records + (size_t)n * 8;
+                    r[0] = cta; r[1] = p.item; r[2] = p.h; r[3] = p.pr; r[4] = p.j0; r[5] = p.j1; r[6] = p.slot; r[7] = p.two;
+                }
+                ++n;
             }
-            ++n;
         }
-    }
+    };
+    if (n_items > kMaxInline) walk(PieceIter<true>()); else walk(PieceIter<false>());
     return n;
 }
 
@@ -858,6 +951,15 @@ ff_status ff_debug_set_trace(ff_cache* c, void* buf, int32_t cap) {
     if (!c || cap < 0) return FF_ERR_INVALID_ARG;
     c->trace = static_cast<unsigned long long*>(buf);
     c->trace_cap = buf ? cap : 0;
+    return FF_OK;
+}
+
+/* Test hook for the error path of a launch: the nth launch site from now (1 = the next one; publish, attention and
+ * merge launches each count as one site, also on a bookkeeping-only cache) reports a failure on the host without
+ * launching anything, and the call it belongs to returns FF_ERR_CUDA.  nth = 0 disarms the hook. */
+ff_status ff_debug_fail_launch(ff_cache* c, int32_t nth) {
+    if (!c || nth < 0) return FF_ERR_INVALID_ARG;
+    c->fail_launch_in = nth;
     return FF_OK;
 }
 

@@ -52,7 +52,9 @@ struct PublishArgs {
     RopeTables tab;
 };
 
-constexpr int kMaxBatch = 8;   // layer-calls of different stages that one attention launch can serve
+constexpr int kMaxInline = 8;   // layer-calls whose descriptors travel as kernel parameters
+constexpr int kMaxBatch = 128;  // layer-calls one attention launch can serve; beyond kMaxInline the descriptors
+                                // are read from a table in device memory (the whole clip of a stage in one launch)
 
 // One layer-call inside an attention launch: its queries, its visible key segments, its output.
 struct AttnItem {
@@ -71,7 +73,7 @@ struct AttnItem {
 // The publishes of one batched layer-call (one kernel launch; blockIdx.y selects the item).
 struct PublishBatch {
     int32_t n;
-    PublishArgs items[kMaxBatch];
+    PublishArgs items[kMaxInline];
 };
 
 struct AttnArgs {
@@ -82,8 +84,10 @@ struct AttnArgs {
     int32_t n_heads, head_dim;
     float scale;         // 1/sqrt(d)
     uint32_t* status;
+    uint32_t launch_tag;      // launch sequence number << 16: or-ed into every error code this launch records
     int32_t n_items;
-    AttnItem items[kMaxBatch];
+    const AttnItem* items_tab;  // n_items > kMaxInline: the descriptors (device memory; host memory while planning)
+    AttnItem items[kMaxInline]; // n_items <= kMaxInline: the descriptors themselves
     // schedule of the tensor-core kernel (filled by attn_tcgen05_plan)
     int32_t n_pairs;          // query-tile pairs over all items and heads
     int32_t n_full;           // whole pairs every CTA handles first (pair r * n_ctas + cta)
@@ -126,12 +130,14 @@ inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 b
 // Launchers (defined in the .cu files).  Each returns the cudaError_t of the launch.
 cudaError_t launch_rope_publish(const PublishArgs& a, int dtype, int sm_count, cudaStream_t s);
 cudaError_t launch_rope_publish_batch(const PublishBatch& b, int dtype, int sm_count, cudaStream_t s);
-cudaError_t launch_attn_simt(const AttnArgs& a, int item, int dtype, cudaStream_t s);
-cudaError_t launch_attn_tcgen05(AttnArgs& a, int n_ctas_max, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
+cudaError_t launch_attn_simt(const AttnArgs& shared, const AttnItem& item, int dtype, cudaStream_t s);
+// Fills the schedule fields of `a` and of the n_items descriptors in `items` (HOST memory: a.items itself, or the
+// host copy of the table for more than kMaxInline items); returns the number of remainder pairs whose pieces need
+// merging afterwards (0 = no merge launch).
+int attn_tcgen05_plan(AttnArgs& a, AttnItem* items, int n_ctas_max);
+// Launches a planned `a`; a.items_tab must be null (inline descriptors) or the DEVICE copy of the planned table.
+cudaError_t launch_attn_tcgen05(const AttnArgs& a, int merge_pairs, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                                 const CUtensorMap& tm_v, cudaStream_t s, int* n_launches);
-// Fills the schedule fields; returns the number of remainder pairs whose pieces need merging afterwards
-// (0 = no merge launch).
-int attn_tcgen05_plan(AttnArgs& a, int n_ctas_max);
 cudaError_t attn_tcgen05_prepare(int head_dim);  // sets the dynamic shared-memory attribute once
 cudaError_t launch_wait_probe(uint32_t* status, unsigned long long limit_ns, cudaStream_t s);
 

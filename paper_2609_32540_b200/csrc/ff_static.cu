@@ -14,7 +14,6 @@
 // streams, or different host threads - race on it.
 #include <cmath>
 #include <mutex>
-#include <vector>
 
 #include "../../include/ff.h"
 #include "ff_internal.h"
@@ -45,13 +44,22 @@ ff_status scratch_address(int device, unsigned char** out) {
     return FF_OK;
 }
 
-void fill_table(std::vector<float2>& tab, size_t at, int first_pos, int n_pos, int n_pairs, double theta) {
-    for (int p = 0; p < n_pos; ++p)
-        for (int j = 0; j < n_pairs; ++j) {
-            const double freq = std::pow(theta, -(double)j / (double)n_pairs);
-            const double ang = (double)(first_pos + p) * freq;
-            tab[at + (size_t)p * n_pairs + j] = make_float2((float)std::cos(ang), (float)std::sin(ang));
-        }
+// Rotary tables written by the device itself, straight into the static array: (cos, sin) of pos * theta^(-j/n),
+// angle and functions in double, each rounded once to float.  No host buffer and no copy are involved, so the
+// call neither blocks the host nor leaves a host pointer behind in a captured stream.
+struct TableJob {
+    float2* dst;       // [n_pos][n_pairs]
+    int first_pos, n_pos, n_pairs;
+};
+__global__ void static_tables_kernel(TableJob f, TableJob y, TableJob x, double theta) {
+    const TableJob job = blockIdx.y == 0 ? f : (blockIdx.y == 1 ? y : x);
+    const int n = job.n_pos * job.n_pairs;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const int p = i / job.n_pairs, j = i - p * job.n_pairs;
+        const double freq = pow(theta, -(double)j / (double)job.n_pairs);
+        const double ang = (double)(job.first_pos + p) * freq;
+        job.dst[i] = make_float2((float)cos(ang), (float)sin(ang));
+    }
 }
 
 }  // namespace
@@ -87,14 +95,12 @@ extern "C" ff_status ff_chunk_attn_static(int32_t n_heads, int32_t head_dim, int
     if (st != FF_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
-    // rotary tables for exactly the positions of this call; the copy from pageable memory is staged before
-    // cudaMemcpyAsync returns, so the vector may go out of scope
-    std::vector<float2> tab(tab_elems);
-    fill_table(tab, tab_at[0], first_frame_pos, n_frames, pairs[0], (double)rope_theta);
-    fill_table(tab, tab_at[1], 0, grid_h, pairs[1], (double)rope_theta);
-    fill_table(tab, tab_at[2], 0, grid_w, pairs[2], (double)rope_theta);
-    if (cudaMemcpyAsync(base, tab.data(), tab_elems * sizeof(float2), cudaMemcpyHostToDevice, s) != cudaSuccess)
-        return FF_ERR_CUDA;
+    // rotary tables for exactly the positions of this call, evaluated on the device
+    float2* t0 = reinterpret_cast<float2*>(base);
+    const TableJob jf{t0 + tab_at[0], first_frame_pos, n_frames, pairs[0]}, jy{t0 + tab_at[1], 0, grid_h, pairs[1]},
+        jx{t0 + tab_at[2], 0, grid_w, pairs[2]};
+    static_tables_kernel<<<dim3(8, 3), 128, 0, s>>>(jf, jy, jx, (double)rope_theta);
+    if (cudaGetLastError() != cudaSuccess) return FF_ERR_CUDA;
 
     PublishArgs p{};
     p.q = q; p.k = k; p.v = v;
@@ -106,7 +112,6 @@ extern "C" ff_status ff_chunk_attn_static(int32_t n_heads, int32_t head_dim, int
     p.first_frame_pos = 0;  // the frame table starts at this call's first frame
     p.frame_pos_stride = 1;
     p.qk_norm = 0; p.qk_norm_eps = 0.f; p.gain_q = nullptr; p.gain_k = nullptr;
-    const float2* t0 = reinterpret_cast<const float2*>(base);
     p.tab.frame = t0 + tab_at[0]; p.tab.row = t0 + tab_at[1]; p.tab.col = t0 + tab_at[2];
     p.tab.pairs_f = pairs[0]; p.tab.pairs_h = pairs[1]; p.tab.pairs_w = pairs[2];
     int sms = 148;
@@ -120,10 +125,10 @@ extern "C" ff_status ff_chunk_attn_static(int32_t n_heads, int32_t head_dim, int
     a.scale = 1.0f / std::sqrt((float)head_dim);
     a.status = nullptr;
     a.n_items = 1;
-    AttnItem& it = a.items[0];
+    AttnItem it{};
     it.out = out; it.q_row0 = 0; it.n_q = (int)n_tok;
     it.segs.n = 1;
     it.segs.row0[0] = 0; it.segs.head_stride[0] = n_tok_pad; it.segs.tokens[0] = (int)n_tok;
-    if (launch_attn_simt(a, 0, dtype, s) != cudaSuccess) return FF_ERR_CUDA;
+    if (launch_attn_simt(a, it, dtype, s) != cudaSuccess) return FF_ERR_CUDA;
     return FF_OK;
 }

@@ -11,9 +11,12 @@
 // from tables the host evaluated in double and rounded to float; each product and each sum is rounded
 // separately (no fused multiply-add), then the result is rounded to nearest-even bf16.
 #include <cuda_bf16.h>
+#include <atomic>
 #include "ff_internal.h"
 
 namespace ffk {
+
+constexpr int kMaxDevices = 64;
 
 __device__ __forceinline__ void rotate(float a, float b, float2 cs, float& r0, float& r1) {
     float t1 = __fmul_rn(a, cs.x);
@@ -195,12 +198,17 @@ namespace {
 // wave, which shows in a kernel this short.
 template <bool kBf16, bool kNorm>
 cudaError_t launch_variant(const PublishBatch& b, int sm_count, cudaStream_t s) {
-    static int per_sm = 0;
+    // resident blocks per SM of this variant on the current device, asked once per device
+    static std::atomic<int> per_sm_of[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = 0;
+    int per_sm = per_sm_of[dev].load(std::memory_order_relaxed);
     if (per_sm == 0) {
         int n = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, rope_publish_kernel<kBf16, kNorm>, 256, 0) != cudaSuccess || n < 1)
             n = 1;
         per_sm = n;
+        per_sm_of[dev].store(n, std::memory_order_relaxed);
     }
     const int elems = kBf16 ? 8 : 4;
     long long blocks = 1;  // per item: at least one pass of rows per block, for the largest item
@@ -220,7 +228,7 @@ cudaError_t launch_variant(const PublishBatch& b, int sm_count, cudaStream_t s) 
 }  // namespace
 
 cudaError_t launch_rope_publish_batch(const PublishBatch& b, int dtype, int sm_count, cudaStream_t s) {
-    if (b.n < 1 || b.n > kMaxBatch) return cudaErrorInvalidValue;
+    if (b.n < 1 || b.n > kMaxInline) return cudaErrorInvalidValue;
     const bool norm = b.items[0].qk_norm != 0;
     if (dtype == 0) return norm ? launch_variant<true, true>(b, sm_count, s) : launch_variant<true, false>(b, sm_count, s);
     return norm ? launch_variant<false, true>(b, sm_count, s) : launch_variant<false, false>(b, sm_count, s);

@@ -71,7 +71,9 @@ __device__ __forceinline__ uint32_t mbar_test_wait(uint64_t* bar, uint32_t parit
 
 // Waits for the phase with the given parity to complete.  Never spins forever: after kWaitLimitNs the
 // code `err` is stored to *status (first error wins) and false is returned; the caller carries on so that the
-// kernel still terminates and releases what it holds.
+// kernel still terminates and releases what it holds.  `err` carries the launch's tag in its upper 16 bits: a
+// wait also gives up early when another wait of the SAME launch has already expired, but an error left behind by
+// an earlier launch (not yet collected by the host) does not shorten this launch's waits.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* status, uint32_t err,
                                           unsigned long long limit_ns = kWaitLimitNs) {
     if (mbar_test_wait(bar, parity)) return true;  // a completed phase is seen without the parking machinery
@@ -80,7 +82,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 15u) == 0) {  // an attempt may park the thread for kSuspendHintNs, so the clock is read often
             // once any wait of the launch has expired, the others give up at their next check
-            if (status && *reinterpret_cast<volatile uint32_t*>(status) != 0u) return false;
+            if (status) {
+                const uint32_t seen = *reinterpret_cast<volatile uint32_t*>(status);
+                if (seen != 0u && (seen >> 16) == (err >> 16)) return false;
+            }
             unsigned long long now = globaltimer_ns();
             if (t0 == 0) {
                 t0 = now;

@@ -40,6 +40,32 @@ def test_fused_qk_norm_head_dim_128_ragged_multi_tile():
     gpu.close()
 
 
+def test_fused_qk_norm_cache_is_within_one_bf16_ulp_of_the_float64_definition():
+    """The bit-exact comparisons above rest on the oracle summing squares in the same order as the kernel (running
+    sums over 16-byte pieces, then a balanced tree).  This one does not: the published K' is compared with
+    normalise -> gain -> rotate written out in float64 here (numpy for the normalisation, the complex-form rotary
+    of the paper definitions), and must agree to one bf16 unit in the last place."""
+    w = W.Workload("norm_f64", 1, 3, 128, 5, 9, 2, 1, 1, 2, 0, 0, "none", 1)
+    eps = 1e-6
+    gpu = Hn.GpuCache(w, O.BF16, attn_impl=1, qk_norm_eps=eps)
+    gq, gk = W.channel_gains(w, 13, 0)
+    assert gpu.cache.ff_cache_set_qk_gain(0, gq.tolist(), gk.tolist(), gpu.stream) == 0
+    q, k, v = W.qkv(w, 13, 0, 0, 0, w.chunk_frames, torch.bfloat16, pre_normalised=False)
+    st, out = gpu.forward(0, 0, 0, w.chunk_frames, 3, q.cuda(), k.cuda(), v.cuda(), [])
+    assert st == 0
+    torch.cuda.synchronize()
+    n = k.shape[0]
+    ck, cv, _ = gpu.read_slot(0, 0, 0, 0, n)
+    x = k.double().numpy()
+    normed = x / np.sqrt((x * x).mean(axis=-1, keepdims=True) + eps) * gk.double().numpy()
+    want = PD.rope_complex(normed, PD.token_positions(w.chunk_frames, 3, w.grid_h, w.grid_w)[:, None, :])
+    got = ck.double().numpy()
+    ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(want), 2.0 ** -126))) - 7)     # bf16: 8 significant bits
+    assert np.all(np.abs(got - want) <= ulp), float((np.abs(got - want) / ulp).max())
+    assert np.array_equal(Hn.bits(cv), Hn.bits(v))
+    gpu.close()
+
+
 def test_qk_norm_off_rejects_gain_and_unit_gain_equals_no_gain():
     gpu = Hn.GpuCache(TINY, O.BF16)
     assert gpu.cache.ff_cache_set_qk_gain(0, [1.0] * TINY.head_dim, None, gpu.stream) == gpu.P.FF_ERR_STATE

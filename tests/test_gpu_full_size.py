@@ -27,6 +27,16 @@ def test_wan1p3b_480p_full_shape():
     gpu.close()
 
 
+def test_wan1p3b_480p_every_row_of_a_steady_state_call():
+    """One steady-state layer-call of config 2 (anchor + two history chunks + own chunk: 15600 keys) compared with
+    the oracle on ALL 4680 rows x 12 heads, not a sample: about half a minute of CPU work for the oracle."""
+    w = W.scaled(W.CONFIGS["wan1p3b_480p"], total_frames=9, n_layers=1)
+    stats, gpu, orc = Hn.run_both(w, O.BF16, attn_impl=1, seed=11, rows_fn=None, check_layers=[0], check_stages=[1],
+                                  pooled=True, check_chunks=[2])
+    assert len(stats) == 1 and stats[0]["max_abs"] > 0
+    gpu.close()
+
+
 def test_wan1p3b_480p_peaked_logits():
     """Same shape with logits x8: O(1) outputs, so a dropped segment or tile cannot hide under the tolerance."""
     w = W.scaled(W.CONFIGS["wan1p3b_480p"], total_frames=9, n_layers=2)
@@ -59,15 +69,15 @@ def test_wan14b_720p_full_shape():
 
 def test_wan1p3b_480p_long_stream():
     """Config 3: the 261-frame stream (87 chunks, 22 anchor publishes, ring and anchor-slot reuse throughout) with
-    all 4 stages on one GPU; the oracle follows one (stage, layer) through the whole stream and compares outputs
+    all 4 stages and all 30 layers on one GPU; the oracle follows one (stage, layer) through the whole stream and compares outputs
     at the start, in the middle and at the end, and the published slot at those chunks."""
-    w = W.scaled(W.CONFIGS["wan1p3b_480p_stream65s"], n_layers=4)
-    assert w.n_chunks == 87
+    w = W.CONFIGS["wan1p3b_480p_stream65s"]
+    assert w.n_chunks == 87 and w.n_layers == 30
     stats, gpu, orc = Hn.run_both(w, O.BF16, attn_impl=1, seed=7, rows_fn=lambda n: W.sample_rows(n, extra=2),
-                                  check_layers=[3], check_stages=[0], pooled=True, check_chunks=[0, 1, 2, 3, 4, 43, 85, 86])
+                                  check_layers=[29], check_stages=[0], pooled=True, check_chunks=[0, 1, 2, 3, 4, 43, 85, 86])
     assert len(stats) == 8
     c = gpu.cache.ff_cache_counters()
-    assert c["layer_calls"] == 87 * 4 * 4 and c["advances"] == 87 * 4 and c["anchor_publishes"] == 22 * 4
+    assert c["layer_calls"] == 87 * 4 * 30 and c["advances"] == 87 * 4 and c["anchor_publishes"] == 22 * 30
     for stage in range(4):
         s = gpu.cache.ff_cache_ring_state(stage, 0)
         assert s["next_chunk"] == 87 and s["head"] == 87 % 3 and s["count"] == 2

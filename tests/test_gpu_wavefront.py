@@ -90,6 +90,36 @@ def test_clip_at_once_ragged_multi_tile():
     gpu.close()
 
 
+def test_whole_clip_in_one_launch_tiny_and_ragged():
+    """group = N_R: every chunk of a stage shares one attention launch per layer.  More layer-calls than travel as
+    launch arguments, so the kernel reads its per-call descriptors from the table in the arena."""
+    w = W.scaled(TINY, total_frames=11, n_anchor_slots=4)
+    assert w.n_chunks == 11
+    for impl, dtype in ((1, O.BF16), (2, O.F32)):
+        stats, gpu, orc = Hn.run_packed_clip(w, w.n_chunks, dtype, attn_impl=impl, seed=2)
+        assert len(stats) == w.n_chunks * w.n_stages * w.n_layers
+        c = gpu.cache.ff_cache_counters()
+        if impl == 1:   # per (stage, layer): two publish launches (8 + 3 calls), one attention launch, at most one merge
+            assert c["kernel_launches"] - c["anchor_publishes"] <= w.n_stages * w.n_layers * 4
+        gpu.close()
+    w = W.Workload("clip_ragged_whole", 2, 3, 128, 9, 23, 2, 2, 2, 19, 2, 6, "bracket", 4)   # 10 chunks, the last short
+    assert w.n_chunks == 10 and w.chunk_frames_of(9) == 1
+    stats, gpu, orc = Hn.run_packed_clip(w, w.n_chunks, O.BF16, attn_impl=1, seed=5, rows_fn=lambda n: W.sample_rows(n, 16, 4))
+    assert len(stats) == w.n_chunks * w.n_stages * w.n_layers
+    gpu.close()
+
+
+def test_whole_81_latent_clip_in_one_launch_at_480p_token_counts():
+    """The paper's worked example at full 480p token counts (27 chunks, H = 5, three anchors per window), one stage
+    and two layers: ONE attention launch per layer over all 27 chunks; sampled rows of every chunk against the
+    chunk-by-chunk oracle, every published slot bit for bit."""
+    w = W.scaled(W.PAPER_480P, n_layers=2, n_stages=1, n_anchor_slots=9)
+    assert w.n_chunks == 27
+    stats, gpu, orc = Hn.run_packed_clip(w, 27, O.BF16, attn_impl=1, seed=9, rows_fn=lambda n: W.sample_rows(n, 3, 9))
+    assert len(stats) == 27 * 2
+    gpu.close()
+
+
 def test_same_stage_batch_needs_enough_slots():
     w = W.scaled(TINY, anchor_policy="none")
     gpu = Hn.GpuCache(w, O.BF16, attn_impl=1, max_batch=4)          # default bank: H + 1 slots

@@ -256,6 +256,11 @@ def _check_schedule(B, n_heads, n_q, n_kv, n_ctas_max=148):
     (2, [64], [128 + 64]), (2, [64, 64], [64, 192]),    # tiny
     (3, [414, 207], [1449, 621]),                       # ragged, short last chunk in one stage
     (1, [129], [1]), (5, [1000] * 8, [3000] * 8),
+    # more layer-calls than travel as launch arguments (descriptor table): a clip's chunks in one launch, with the
+    # warm-up chunks seeing fewer keys and a short last chunk
+    (12, [4680] * 27, [min(i + 1, 6) * 4680 + 3 * 1560 for i in range(27)]),
+    (2, [64] * 9, [64 * min(i + 1, 3) for i in range(9)]),
+    (3, [300] * 40 + [100], [300 * min(i + 1, 4) + 77 for i in range(40)] + [1377]),
 ])
 def test_attention_work_distribution_covers_everything_once(B, n_heads, n_q, n_kv):
     for n_ctas in (148, 7, 1):
@@ -298,6 +303,66 @@ def test_same_stage_batches_follow_the_slot_rule(B):
     assert c.ff_batch_forward_attn(0, [item(1, 3), item(1, 4), item(1, 5)]) == B.FF_OK
     assert c.ff_cache_ring_state(1, 0)["slot_chunk"][0] == 5
     c.close()
+
+
+def test_a_refused_launch_leaves_the_tables_and_counters_untouched(B):
+    """Host-injected launch failure (no GPU involved): whichever launch site of a call fails, the call returns
+    FF_ERR_CUDA and the ring table, the anchor table and the counters are what they were; the same call then
+    succeeds."""
+    w = W.scaled(W.CONFIGS["tiny"], n_stages=2)
+    c = _dry_cache(B, w)
+
+    def snapshot():
+        return ([c.ff_cache_ring_state(s, 0) for s in range(w.n_stages)], c.ff_cache_anchor_state(0), c.ff_cache_counters())
+
+    before = snapshot()
+    assert c.ff_debug_fail_launch(1) == B.FF_OK
+    assert c.ff_anchor_publish(0, 3, 0, 16, 16) == B.FF_ERR_CUDA
+    assert B.ff_last_cuda_error() != 0 and snapshot() == before
+    assert c.ff_anchor_publish(0, 3, 0, 16, 16) == B.FF_OK
+    before = snapshot()
+    # a single call has two launch sites (publish, attention); a batch of two stages has the same two
+    for nth in (1, 2):
+        assert c.ff_debug_fail_launch(nth) == B.FF_OK
+        assert c.ff_chunk_forward_attn(1, 0, 0, 1, 0, 16, 16, 16, [0], 16) == B.FF_ERR_CUDA
+        assert snapshot() == before
+        assert c.ff_cache_advance(1) == B.FF_ERR_STATE           # the chunk was never recorded as published
+    items = [dict(stage=s, chunk_index=0, n_frames=1, first_frame_pos=0, q=16, k=16, v=16, out=16, anchor_slots=[0])
+             for s in (1, 0)]
+    assert c.ff_debug_fail_launch(2) == B.FF_OK
+    assert c.ff_batch_forward_attn(0, items) == B.FF_ERR_CUDA and snapshot() == before
+    assert c.ff_batch_forward_attn(0, items) == B.FF_OK
+    after = snapshot()
+    assert after[2]["layer_calls"] == before[2]["layer_calls"] + 2
+    assert [st["slot_chunk"][0] for st in after[0]] == [0, 0]
+    assert c.ff_cache_advance(1) == B.FF_OK and c.ff_cache_advance(0) == B.FF_OK
+    assert c.ff_debug_fail_launch(-1) == B.FF_ERR_INVALID_ARG
+    c.close()
+
+
+def test_whole_clip_of_a_stage_in_one_batch(B):
+    """All 27 chunks of the 81-latent clip as ONE batched call per layer (bookkeeping-only cache): needs H + 27 bank
+    slots and 27 query regions; the later chunks see the earlier ones' token counts, the last chunk may be short."""
+    w = W.scaled(W.PAPER_480P, n_layers=2, n_stages=1, grid_h=2, grid_w=4, total_frames=80)   # 26 chunks of 3 + one of 2
+    N, H = w.n_chunks, w.history_chunks
+    assert N == 27
+    kw = dict(n_layers=w.n_layers, n_heads=w.n_heads, head_dim=w.head_dim, grid_h=w.grid_h, grid_w=w.grid_w,
+              chunk_frames=w.chunk_frames, n_stages=1, history_chunks=H, n_anchor_slots=0, max_visible_anchors=0,
+              device=B.FF_DEVICE_NONE)
+    c = B.Cache(B.make_config(**kw, ring_slots=H + N, max_batch=N), None, 0)
+    items = [dict(stage=0, chunk_index=i, n_frames=w.chunk_frames_of(i), first_frame_pos=3 * i, q=16, k=16, v=16, out=16)
+             for i in range(N)]
+    for l in range(w.n_layers):
+        assert c.ff_batch_forward_attn(l, items) == B.FF_OK
+    st = c.ff_cache_ring_state(0, 1)
+    assert st["slot_chunk"][:N] == list(range(N)) and st["slot_tokens"][N - 1] == 2 * w.tokens_per_frame
+    for i in range(N):
+        assert c.ff_cache_advance(0) == B.FF_OK
+    assert c.ff_cache_counters()["layer_calls"] == 2 * N
+    c.close()
+    small = B.Cache(B.make_config(**kw, ring_slots=H + N, max_batch=8), None, 0)
+    assert small.ff_batch_forward_attn(0, items) == B.FF_ERR_UNSUPPORTED      # more calls than query regions
+    small.close()
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

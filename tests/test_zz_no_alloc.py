@@ -4,8 +4,10 @@ ff_chunk_attn_static serves callers that get device buffers handed to them but m
 themselves (a plug-in inside a server whose pool belongs to the framework, a loop that cannot take cudaMalloc's
 implicit synchronisation).  Its scratch is one fixed device array inside the library, shared by all calls, which
 still holds the previous call's data when the next call starts - so the check runs two different calls back to
-back and compares each with ff_chunk_forward_attn on a fresh cache (chunk 0, no anchors, CUDA-core kernel),
-which computes the same thing out of a caller-provided arena.
+back and compares each (a) with the CPU oracle's first-chunk call (chunk 0, empty bank, no anchors), every row,
+within the tolerance of the other parity tests, and (b) with ff_chunk_forward_attn on a fresh cache (CUDA-core
+kernel), which computes the same thing out of a caller-provided arena.  A third check reads the device's free
+memory around a warm call: the call must not change it.
 
 Collected last on purpose: a failure here cannot hide the result of any other test in a run that stops at the
 first failure.  It passes alone in a fresh process and after the other tests.
@@ -48,12 +50,40 @@ def test_static_scratch_entry_point_matches_arena_entry_point_twice(dtype):
                                     dtype, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), stream)
         assert st == B.FF_OK, st
         torch.cuda.synchronize()
+        # (a) the oracle, written from the definition: rotate, publish, attend over the chunk's own keys
+        orc = Hn.make_oracle(w, dtype)
+        so, truth = orc.chunk_forward(0, 0, 0, w.chunk_frames, pos, q.float().cpu().numpy(), k.float().cpu().numpy(),
+                                      v.float().cpu().numpy(), [])
+        assert so == O.OK
+        Hn.compare_outputs(out, truth, dtype, f"static entry point, {w.name}")
+        # (b) the arena entry point: same kernels; its rotary tables are evaluated on the host, this one's on the
+        # device, so a rotated element may differ in its last bit
         want = _reference(w, dtype, q, k, v, pos)
-        assert torch.isfinite(out.float()).all()
         err = (out.float() - want.float()).abs()
         tol = Hn.F32_ABS_TOL if dtype == O.F32 else Hn.ABS_MAX_TOL
         assert err.max().item() <= tol, err.max().item()
-        assert torch.equal(out, want)      # same kernels, same arithmetic: in fact bit-identical
+
+
+def test_static_scratch_entry_point_leaves_free_device_memory_unchanged():
+    """The claim "allocates nothing", measured: free device memory before and after a call on a warm library (the
+    first call on a device may load the kernels' module) is the same to the byte."""
+    from paper_2609_32540_b200 import binding as B
+    w = W.Workload("na3", 1, 2, 64, 8, 8, 1, 1, 0, 1, 0, 0, "none", 1)
+    q, k, v = (t.cuda() for t in W.qkv(w, 3, 0, 0, 0, 1, torch.bfloat16))
+    out = torch.empty_like(q)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def call():
+        assert B.ff_chunk_attn_static(w.n_heads, w.head_dim, w.grid_h, w.grid_w, 1, 0, w.rope_theta, B.FF_BF16,
+                                      q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), stream) == B.FF_OK
+        torch.cuda.synchronize()
+
+    call()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        call()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, (free0, free1)
 
 
 def test_static_scratch_entry_point_rejects_what_does_not_fit():
