@@ -602,6 +602,150 @@ def measure_adjacent_steps(P, dev, local: int, hbm_peak_gbs: float) -> dict:
     return out
 
 
+def pipeline_run(P, base: W.Workload, world: int, rank: int, steps: int, warmup: int, device_index, group=None) -> dict:
+    """Stage-per-rank renderer wavefront (Alg. 1 Phase B): `world` ranks, rank r owns the S / world denoising stages
+    r * S/world .. (r+1) * S/world - 1 counted from the noisiest, each in a cache of its own on its own device; a
+    chunk's latent is handed from rank to rank point to point (torch.distributed isend / recv), the banks never
+    move.  world = 1 is the chunk-major order on one device.  Runs `warmup` chunks untimed, then times `steps`
+    chunks from a barrier until this rank has finished its last one (pipeline fill and drain included).
+    device_index None = bookkeeping-only caches and CPU latents: the same code path without a GPU (tests)."""
+    import torch.distributed as dist
+    from paper_2609_32540_b200 import wavefront as Wf
+    S = base.n_stages
+    assert S % world == 0, "the ranks must share the denoising stages equally"
+    n_local = S // world
+    dry = device_index is None
+    n_total = warmup + steps
+    w = W.scaled(base, n_stages=n_local, total_frames=(n_total + 2) * base.chunk_frames, clip_anchor_pos=False,
+                 max_frame_pos=(n_total + 12) * base.chunk_frames + 16,
+                 n_anchor_slots=max(base.n_anchor_slots, 2 * base.visible_anchors + 1))
+    dev = torch.device("cpu") if dry else torch.device(f"cuda:{device_index}")
+    cfg = P.make_config(n_layers=w.n_layers, n_heads=w.n_heads, head_dim=w.head_dim, grid_h=w.grid_h, grid_w=w.grid_w,
+                        chunk_frames=w.chunk_frames, n_stages=n_local, history_chunks=w.history_chunks,
+                        n_anchor_slots=w.n_anchor_slots, max_visible_anchors=w.visible_anchors, dtype=P.FF_BF16,
+                        attn_impl=P.FF_ATTN_TCGEN05, max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta,
+                        device=P.FF_DEVICE_NONE if dry else device_index)
+    if dry:
+        arena, cache, stream = None, P.Cache(cfg, None, 0), 0
+        io = P.make_io([(16, 16, 16, 16)] * w.n_layers)
+        ak_ptr = av_ptr = 16
+    else:
+        nbytes = P.ff_cache_query_bytes(cfg)
+        arena = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        cache = P.Cache(cfg, arena.data_ptr(), nbytes)
+        stream = torch.cuda.current_stream().cuda_stream
+        sets = []
+        for sidx in range(N_IO):
+            q, k, v = W.qkv(w, 6, sidx, rank, 0)
+            sets.append((q.to(dev), k.to(dev), v.to(dev), torch.empty_like(q, device=dev)))
+        io = P.make_io([(sets[l % N_IO][0].data_ptr(), sets[l % N_IO][1].data_ptr(), sets[l % N_IO][2].data_ptr(),
+                         sets[l % N_IO][3].data_ptr()) for l in range(w.n_layers)])
+        ak, av = (t.to(dev) for t in W.anchor_kv(w, 6, 0, 0))
+        ak_ptr, av_ptr = ak.data_ptr(), av.data_ptr()
+    # the chunk's latent: 16 channels on a grid twice as fine as the token grid, float32; the velocity stands in
+    # for the forward's prediction
+    n_lat = w.chunk_frames * 16 * (2 * w.grid_h) * (2 * w.grid_w)
+    like = torch.zeros(n_lat, dtype=torch.float32, device=dev)
+    velocity = torch.ones(n_lat, dtype=torch.float32 if dry else torch.bfloat16, device=dev)
+    levels = [(P.ff_plan_sigma(S - rank * n_local - j, S), P.ff_plan_sigma(S - rank * n_local - j - 1, S))
+              for j in range(n_local)]
+    stages = Wf.RendererStages(cache, P.binding, levels, io, velocity, stream, dry)
+    published = set()
+
+    def run_node(i, x):
+        ids = W.visible_anchor_ids(w, i)
+        for m in ids:       # every rank keeps its own copy of the clean anchor bank
+            if m not in published:
+                published.add(m)
+                for l in range(w.n_layers):
+                    st = cache.ff_anchor_publish(W.anchor_slot(w, m), W.anchor_frame_pos(w, m), l, ak_ptr, av_ptr, stream)
+                    assert st == 0, st
+        return stages.run_node(i, w.chunk_frames, i * w.chunk_frames, [W.anchor_slot(w, m) for m in ids], x)
+
+    delivered = []
+    noise = torch.full_like(like, 1.0)
+
+    def make_rank(n_chunks, first):
+        return Wf.StageRank(rank, world, n_chunks, like, obtain=(lambda i: noise.clone()) if rank == 0 else None,
+                            run_node=run_node, deliver=lambda i, x: delivered.append(i), group=group, first_chunk=first)
+
+    def barrier():
+        if not dry:
+            torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier(group=group)
+
+    make_rank(warmup, 0).run()
+    barrier()
+    c0 = cache.ff_cache_counters()
+    t0 = time.perf_counter()
+    if not dry:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+    stats = make_rank(steps, warmup).run()
+    if not dry:
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+    else:
+        ms = 1e3 * (time.perf_counter() - t0)
+    c1 = cache.ff_cache_counters()
+    st, word = cache.ff_cache_status(stream)
+    assert st == 0 and word == 0, (st, hex(word))
+    flops_rank = sum(chunk_flops(w, warmup + j) for j in range(steps))     # this rank's stages only
+    res = dict(rank=rank, ms=ms, chunks=stats.chunks, sent=stats.sent, received=stats.received,
+               layer_calls=c1["layer_calls"] - c0["layer_calls"], advances=c1["advances"] - c0["advances"],
+               gpu_launches=c1["kernel_launches"] - c0["kernel_launches"], delivered=list(delivered),
+               flops=flops_rank, stages_per_rank=n_local, latent_bytes=n_lat * 4, n_q=w.chunk_frames * w.tokens_per_frame,
+               n_kv=w.steady_n_kv())
+    cache.close()
+    return res
+
+
+def run_wavefront_mode(args):
+    """bench.py --mode wavefront: the stage-per-GPU pipeline on --gpus ranks (torchrun), one JSON line from rank 0."""
+    import torch.distributed as dist
+    import paper_2609_32540_b200 as P
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+    base = W.CONFIGS[args.workload]
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    res = pipeline_run(P, base, world, rank, args.steps, max(args.warmup, base.history_chunks + 2), local)
+    clocks = sampler.stop() if rank == 0 else {}
+    ms = max_over_ranks(res["ms"], world, dev)
+    flops = res["flops"]
+    launches = res["gpu_launches"]
+    if world > 1:
+        t = torch.tensor([flops, float(launches)], device=dev, dtype=torch.float64)
+        dist.all_reduce(t)
+        flops, launches = float(t[0].item()), int(t[1].item())
+    if rank == 0:
+        peaks = read_peaks()
+        value = flops / (ms * 1e-3) / 1e12
+        cfg = config_dict(base, world, args.workload)
+        cfg["parallelism"] = f"stage pipeline x{world} ({res['stages_per_rank']} denoising stage(s) per rank)"
+        line = dict(metric="chunk_attn_tflops", value=value, unit="TFLOP/s", n_gpus=world, steps=args.steps,
+                    warmup=max(args.warmup, base.history_chunks + 2), ms_per_step=ms / args.steps, higher_is_better=True,
+                    scaling="pipeline", vs_baseline=None, dtype="bf16", data="synthetic", mode="wavefront", config=cfg,
+                    chunks_per_s=args.steps / (ms * 1e-3), clocks=clocks, gpu_launches=launches,
+                    pct_of_measured_bf16_peak=100.0 * value / world / peaks["burst"],
+                    latent_bytes_per_hop=res["latent_bytes"],
+                    note=("timed from a barrier until the slowest rank has finished its last chunk: pipeline fill and "
+                          "drain included; with one rank this is the chunk-major order plus the Euler updates"))
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def run_gpu(args):
     import torch.distributed as dist
     import paper_2609_32540_b200 as P
@@ -703,8 +847,9 @@ def run_gpu(args):
         step(chunk); chunk += 1
     prof = cache.ff_cache_profile_end(stream)
     attn_flops_per_launch = w.flops_per_call()
-    attn_ms = prof["attn_ms"] / max(prof["attn_launches"], 1)
-    publish_ms = prof["publish_ms"] / max(prof["publish_launches"], 1)
+    # per layer-call: one publish launch, and one attention launch followed (when pairs were split) by a merge launch
+    attn_ms = prof["attn_ms"] / calls
+    publish_ms = prof["publish_ms"] / calls
     attn_tflops = attn_flops_per_launch / (attn_ms * 1e-3) / 1e12
     elem = 2
     publish_bytes = 6 * w.chunk_frames * w.tokens_per_frame * w.n_heads * w.head_dim * elem  # read q,k,v; write q',k',v
@@ -780,7 +925,7 @@ def run_gpu(args):
                       achieved=attn_tflops, peak=peaks["sustained"],
                       unit="TFLOP/s", frac=attn_tflops / peaks["sustained"], frac_of_burst_peak=attn_tflops / peaks["burst"],
                       peak_source=f"{peaks['source']} bf16 GEMM, sustained (kernel timed inside a long step)",
-                      ms_per_launch=attn_ms, launches_timed=prof["attn_launches"],
+                      ms_per_launch=attn_ms, layer_calls_timed=calls, launches_timed=prof["attn_launches"],
                       flops_per_launch=attn_flops_per_launch, **ncu_traffic(args.workload),
                       algorithmic_bytes_per_launch=attn_algorithmic_bytes(w),
                       publish=dict(bound="hbm", achieved=publish_gbs, peak=peaks["hbm_gbs"], unit="GB/s",
@@ -830,9 +975,14 @@ def main():
     ap.add_argument("--stream", action="store_true",
                     help="extra: also run the workload's whole stream once from empty banks and report its wall time")
     ap.add_argument("--skip-extra", action="store_true", help="skip the extra measurement at the paper's budget")
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "wavefront"],
+                    help="replicas (default, the headline): every rank runs the whole path on its own GPU; wavefront: "
+                         "the paper's stage-per-GPU pipeline over --gpus ranks (1, 2 or 4 for four stages)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.mode == "wavefront":
+        run_wavefront_mode(args)
     else:
         run_gpu(args)
 

@@ -72,7 +72,10 @@ struct SmemLayout {
 // per row and half tile, 4 lanes per clock), so moving a quarter of them away shortens their exp phase; the step
 // runs on the GPU's power cap, where the extra FMA work costs clock: measured on the 480p shape over 20-step runs,
 // 0: 53.4 ms per step, 4: 52.5, 3: 52.8, 2: 53.2.
-constexpr int kPolyEvery = 4;
+#ifndef FF_POLY_EVERY
+#define FF_POLY_EVERY 4
+#endif
+constexpr int kPolyEvery = FF_POLY_EVERY;
 
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float d;

@@ -50,7 +50,7 @@ class StageRank:
 
     def __init__(self, rank: int, n_stages: int, n_chunks: int, like: torch.Tensor, *,
                  obtain: Optional[Callable[[int], torch.Tensor]], run_node: Callable[[int, torch.Tensor], torch.Tensor],
-                 deliver: Optional[Callable[[int, torch.Tensor], None]] = None, group=None):
+                 deliver: Optional[Callable[[int, torch.Tensor], None]] = None, group=None, first_chunk: int = 0):
         if not 0 <= rank < n_stages:
             raise ValueError("rank outside the stage range")
         if rank == 0 and obtain is None:
@@ -59,6 +59,7 @@ class StageRank:
         self.stage = n_stages - rank          # k in the paper's numbering (S .. 1)
         self.like, self.group = like, group
         self.obtain, self.run_node, self.deliver = obtain, run_node, deliver
+        self.first_chunk = first_chunk        # chunks first_chunk .. first_chunk + n_chunks - 1 (banks may be warm)
         self.stats = WavefrontStats()
 
     def run(self) -> WavefrontStats:
@@ -67,6 +68,7 @@ class StageRank:
             i = n - self.rank
             if not 0 <= i < self.n_chunks:
                 continue
+            i += self.first_chunk
             if self.rank == 0:
                 x = self.obtain(i)
             else:
@@ -87,6 +89,44 @@ class StageRank:
         if pending is not None:
             pending.wait()
         return self.stats
+
+
+class RendererStages:
+    """What one rank of the stage-per-GPU renderer does with a chunk (Alg. 1 Phase B, "Read / Evaluate / Step /
+    Write in place" on the rank that owns stage k): for each denoising stage the rank owns - one when there are as
+    many ranks as stages, all S on a single rank, which is then the chunk-major order - every layer's chunk
+    attention against the rank's own bank, Tail_H, and the Euler update of the chunk's latent.
+
+    cache: a Cache created with n_stages = the number of stages this rank owns (bank index n_local-1 is the
+    noisiest of them).  levels: per owned stage, in the order they run, (sigma_k, sigma_{k-1}).  io: ff_layer_io
+    array of n_layers entries (device pointers of the layer inputs; the projections that would produce them are
+    outside this library).  velocity: tensor shaped like the latent standing in for the forward's prediction.
+    With a bookkeeping-only cache (no device) the calls are validated and counted and the update runs on the
+    latent's own device with torch: the plumbing can be exercised on CPU ranks."""
+
+    def __init__(self, cache, binding, levels, io, velocity: torch.Tensor, stream: int = 0, dry: bool = False):
+        self.cache, self.B, self.levels, self.io = cache, binding, list(levels), io
+        self.velocity, self.stream, self.dry = velocity, stream, dry
+        self.layer_calls = 0
+
+    def run_node(self, chunk: int, n_frames: int, first_frame_pos: int, anchor_slots, x: torch.Tensor) -> torch.Tensor:
+        B = self.B
+        n_local = len(self.levels)
+        for j, (sigma_k, sigma_km1) in enumerate(self.levels):
+            st = self.cache.ff_sched_run_node(n_local - 1 - j, chunk, n_frames, first_frame_pos, list(anchor_slots),
+                                              self.io, self.stream)
+            if st != B.FF_OK:
+                raise B.FFError(st, f"ff_sched_run_node(chunk {chunk}, local stage {n_local - 1 - j})")
+            self.layer_calls += self.cache.cfg.n_layers
+            if self.dry:
+                x = x - (sigma_k - sigma_km1) * self.velocity.to(x.dtype)
+            else:
+                code = {torch.float32: B.FF_F32, torch.bfloat16: B.FF_BF16}
+                st = B.ff_euler_step(x.data_ptr(), self.velocity.data_ptr(), sigma_k, sigma_km1, x.numel(),
+                                     code[x.dtype], code[self.velocity.dtype], x.data_ptr(), self.stream)
+                if st != B.FF_OK:
+                    raise B.FFError(st, "ff_euler_step")
+        return x
 
 
 @dataclass

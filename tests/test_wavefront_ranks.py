@@ -131,6 +131,51 @@ def test_a_rank_that_dies_between_steps_ends_the_others_with_an_error():
     assert by_rank[0][1] == "error"
 
 
+def _bench_rank_main(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world, timeout=timedelta(seconds=20))
+    try:
+        import bench
+        import ff_workloads as W
+        import paper_2609_32540_b200 as P
+        w = W.scaled(W.CONFIGS["tiny"], n_stages=4, n_layers=3)
+        res = bench.pipeline_run(P, w, world, rank, steps=5, warmup=4, device_index=None)
+        q.put((rank, "ok", res))
+    except Exception as e:  # noqa: BLE001
+        q.put((rank, "error", f"{type(e).__name__}: {e}"[:200]))
+    finally:
+        try:
+            dist.destroy_process_group()
+        except Exception:  # noqa: BLE001
+            pass
+
+
+@pytest.mark.parametrize("world", [1, 2])
+def test_bench_wavefront_mode_runs_the_same_code_on_cpu_ranks(world):
+    """bench.py --mode wavefront, as launched on GPUs, is pipeline_run on every rank; here the same function runs on
+    gloo ranks over bookkeeping-only caches: four denoising stages shared by the ranks, every rank's call sequence
+    accepted by its own cache, the latents handed on in order, the clean chunks delivered by the last rank."""
+    from paper_2609_32540_b200 import build
+    build.build()
+    port = _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_bench_rank_main, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=180) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+    for rank, status, r in res:
+        assert status == "ok", r
+        n_local = 4 // world
+        assert r["stages_per_rank"] == n_local and r["chunks"] == 5
+        assert r["layer_calls"] == 5 * n_local * 3 and r["advances"] == 5 * n_local
+        assert r["sent"] == (5 if rank < world - 1 else 0) and r["received"] == (5 if rank > 0 else 0)
+        assert r["delivered"] == (list(range(9)) if rank == world - 1 else [])   # warm-up chunks included
+        assert r["flops"] > 0 and r["ms"] > 0
+
+
 def test_clip_plan_follows_the_papers_windows_and_guards_slot_reuse():
     from paper_2609_32540_b200 import build, wavefront as Wf
     build.build()
