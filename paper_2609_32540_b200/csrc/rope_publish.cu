@@ -71,13 +71,29 @@ __device__ __forceinline__ uint4 rotate_pack_piece(const float (&x)[kBf16 ? 8 : 
 // tree over the row's pieces (xor-butterfly: every lane ends with the same value), mean by an exact power of
 // two, correctly rounded sqrt and division, then per element one rounded product with the inverse and one
 // with the channel's gain.
+// The normalisation is split in three so that the expensive part runs once per row instead of once per lane:
+// row_sum_squares leaves the row's sum of squares in every lane of the row; then ONE lane per row and tensor
+// evaluates 1/sqrt(mean + eps) (inv_rms_shared: the up to four sums a lane holds - two rows in flight, K and Q -
+// are dealt out to the row's first four lanes, each evaluates one, and the results are handed back by shuffle);
+// scale_row applies it.  The values are the same as if every lane had evaluated its own.
 template <int E>
-__device__ __forceinline__ void rms_normalise(float (&x)[E], const float (&gain)[E], int ppr, float inv_d, float eps) {
+__device__ __forceinline__ float row_sum_squares(const float (&x)[E], int ppr) {
     float acc = __fmul_rn(x[0], x[0]);
 #pragma unroll
     for (int e = 1; e < E; ++e) acc = __fadd_rn(acc, __fmul_rn(x[e], x[e]));
     for (int off = 1; off < ppr; off <<= 1) acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
-    const float inv = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fmul_rn(acc, inv_d), eps)));
+    return acc;
+}
+__device__ __forceinline__ void inv_rms_shared(float (&acc)[4], int ppr, float inv_d, float eps) {
+    const int lane = threadIdx.x & 31, row_lane0 = lane & ~(ppr - 1);
+    const int j = lane & 3;
+    const float mine = j == 0 ? acc[0] : (j == 1 ? acc[1] : (j == 2 ? acc[2] : acc[3]));
+    const float inv = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fmul_rn(mine, inv_d), eps)));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i] = __shfl_sync(0xffffffffu, inv, row_lane0 + i);
+}
+template <int E>
+__device__ __forceinline__ void scale_row(float (&x)[E], const float (&gain)[E], float inv) {
 #pragma unroll
     for (int e = 0; e < E; ++e) x[e] = __fmul_rn(__fmul_rn(x[e], inv), gain[e]);
 }
@@ -155,14 +171,35 @@ __global__ void __launch_bounds__(256) rope_publish_kernel(const __grid_constant
                 if (qin) qv[u] = __ldg(qin + src);
             }
         }
+        // with the normalisation both rows are unpacked and normalised first (their inverse RMS values are evaluated
+        // together); without it each row is unpacked where it is rotated, which keeps fewer registers live
+        float kxs[kNorm ? 2 : 1][kElemsPerPiece], qxs[kNorm ? 2 : 1][kElemsPerPiece];
+        if constexpr (kNorm) {   // executed by every lane: rows without data carry zeros
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                unpack_piece<kBf16>(kv[u], kxs[u]);
+                unpack_piece<kBf16>(qv[u], qxs[u]);
+            }
+            float acc[4];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                acc[2 * u] = row_sum_squares<kElemsPerPiece>(kxs[u], ppr);
+                acc[2 * u + 1] = qin ? row_sum_squares<kElemsPerPiece>(qxs[u], ppr) : 0.f;
+            }
+            inv_rms_shared(acc, ppr, inv_d, a.qk_norm_eps);
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                scale_row<kElemsPerPiece>(kxs[u], gain_k, acc[2 * u]);
+                if (qin) scale_row<kElemsPerPiece>(qxs[u], gain_q, acc[2 * u + 1]);
+            }
+        }
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
-            float kx[kElemsPerPiece], qx[kElemsPerPiece];
-            unpack_piece<kBf16>(kv[u], kx);
-            unpack_piece<kBf16>(qv[u], qx);
-            if constexpr (kNorm) {   // executed by every lane: rows without data carry zeros
-                rms_normalise<kElemsPerPiece>(kx, gain_k, ppr, inv_d, a.qk_norm_eps);
-                if (qin) rms_normalise<kElemsPerPiece>(qx, gain_q, ppr, inv_d, a.qk_norm_eps);
+            float (&kx)[kElemsPerPiece] = kxs[kNorm ? u : 0];
+            float (&qx)[kElemsPerPiece] = qxs[kNorm ? u : 0];
+            if constexpr (!kNorm) {
+                unpack_piece<kBf16>(kv[u], kx);
+                unpack_piece<kBf16>(qv[u], qx);
             }
             if (!live[u]) continue;
             const int t = tt[u], h = hh[u];
