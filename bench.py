@@ -280,7 +280,7 @@ def measure_paper_budget(P, dev, local: int, steps: int = 3) -> dict:
         cfg = P.make_config(n_layers=w.n_layers, n_heads=w.n_heads, head_dim=w.head_dim, grid_h=w.grid_h,
                             grid_w=w.grid_w, chunk_frames=w.chunk_frames, n_stages=w.n_stages,
                             history_chunks=w.history_chunks, n_anchor_slots=w.n_anchor_slots,
-                            max_visible_anchors=w.visible_anchors, dtype=P.FF_BF16, attn_impl=P.FF_ATTN_TCGEN05,
+                            max_visible_anchors=w.visible_anchors, dtype=P.FF_BF16, attn_impl=P.FF_ATTN_AUTO,
                             max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta, device=local,
                             frame_pos_stride=w.frame_pos_stride, allow_republish=int(w.allow_republish))
         nbytes = P.ff_cache_query_bytes(cfg)
@@ -349,7 +349,7 @@ def measure_wavefront(P, dev, local: int, workload: str, steps: int) -> dict:
     cfg = P.make_config(n_layers=w.n_layers, n_heads=w.n_heads, head_dim=w.head_dim, grid_h=w.grid_h, grid_w=w.grid_w,
                         chunk_frames=w.chunk_frames, n_stages=w.n_stages, history_chunks=w.history_chunks,
                         n_anchor_slots=w.n_anchor_slots, max_visible_anchors=w.visible_anchors, dtype=P.FF_BF16,
-                        attn_impl=P.FF_ATTN_TCGEN05, max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta,
+                        attn_impl=P.FF_ATTN_AUTO, max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta,
                         device=local)
     nbytes = P.ff_cache_query_bytes(cfg)
     arena = torch.empty(nbytes, dtype=torch.uint8, device=dev)
@@ -420,7 +420,7 @@ def measure_clip_at_once(P, dev, local: int, group: int = 27) -> dict:
     cfg = P.make_config(n_layers=w.n_layers, n_heads=w.n_heads, head_dim=w.head_dim, grid_h=w.grid_h, grid_w=w.grid_w,
                         chunk_frames=w.chunk_frames, n_stages=1, history_chunks=w.history_chunks,
                         n_anchor_slots=w.n_anchor_slots, max_visible_anchors=w.visible_anchors, dtype=P.FF_BF16,
-                        attn_impl=P.FF_ATTN_TCGEN05, max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta,
+                        attn_impl=P.FF_ATTN_AUTO, max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta,
                         device=local, ring_slots=w.history_chunks + group, max_batch=group)
     nbytes = P.ff_cache_query_bytes(cfg)
     arena = torch.empty(nbytes, dtype=torch.uint8, device=dev)
@@ -477,7 +477,7 @@ def measure_peaked_logits(P, dev, local: int, workload: str, steps: int, logit_g
     cfg = P.make_config(n_layers=w.n_layers, n_heads=w.n_heads, head_dim=w.head_dim, grid_h=w.grid_h, grid_w=w.grid_w,
                         chunk_frames=w.chunk_frames, n_stages=w.n_stages, history_chunks=w.history_chunks,
                         n_anchor_slots=w.n_anchor_slots, max_visible_anchors=w.visible_anchors, dtype=P.FF_BF16,
-                        attn_impl=P.FF_ATTN_TCGEN05, max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta,
+                        attn_impl=P.FF_ATTN_AUTO, max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta,
                         device=local)
     nbytes = P.ff_cache_query_bytes(cfg)
     arena = torch.empty(nbytes, dtype=torch.uint8, device=dev)
@@ -543,7 +543,7 @@ def measure_adjacent_steps(P, dev, local: int, hbm_peak_gbs: float) -> dict:
         cfg = P.make_config(n_layers=w.n_layers, n_heads=w.n_heads, head_dim=w.head_dim, grid_h=w.grid_h,
                             grid_w=w.grid_w, chunk_frames=w.chunk_frames, n_stages=w.n_stages,
                             history_chunks=w.history_chunks, n_anchor_slots=w.n_anchor_slots,
-                            max_visible_anchors=w.visible_anchors, dtype=P.FF_BF16, attn_impl=P.FF_ATTN_TCGEN05,
+                            max_visible_anchors=w.visible_anchors, dtype=P.FF_BF16, attn_impl=P.FF_ATTN_AUTO,
                             max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta, device=local, qk_norm=norm)
         nbytes = P.ff_cache_query_bytes(cfg)
         arena = torch.empty(nbytes, dtype=torch.uint8, device=dev)
@@ -623,7 +623,7 @@ def pipeline_run(P, base: W.Workload, world: int, rank: int, steps: int, warmup:
     cfg = P.make_config(n_layers=w.n_layers, n_heads=w.n_heads, head_dim=w.head_dim, grid_h=w.grid_h, grid_w=w.grid_w,
                         chunk_frames=w.chunk_frames, n_stages=n_local, history_chunks=w.history_chunks,
                         n_anchor_slots=w.n_anchor_slots, max_visible_anchors=w.visible_anchors, dtype=P.FF_BF16,
-                        attn_impl=P.FF_ATTN_TCGEN05, max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta,
+                        attn_impl=P.FF_ATTN_AUTO, max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta,
                         device=P.FF_DEVICE_NONE if dry else device_index)
     if dry:
         arena, cache, stream = None, P.Cache(cfg, None, 0), 0
@@ -769,7 +769,7 @@ def run_gpu(args):
     cfg = P.make_config(n_layers=w.n_layers, n_heads=w.n_heads, head_dim=w.head_dim, grid_h=w.grid_h, grid_w=w.grid_w,
                         chunk_frames=w.chunk_frames, n_stages=w.n_stages, history_chunks=w.history_chunks,
                         n_anchor_slots=w.n_anchor_slots, max_visible_anchors=w.visible_anchors, dtype=P.FF_BF16,
-                        attn_impl=P.FF_ATTN_TCGEN05, max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta,
+                        attn_impl=P.FF_ATTN_AUTO, max_frame_pos=w.max_frame_pos, rope_theta=w.rope_theta,
                         device=local)
     nbytes = P.ff_cache_query_bytes(cfg)
     arena = torch.empty(nbytes, dtype=torch.uint8, device=dev)
@@ -836,6 +836,9 @@ def run_gpu(args):
     clocks = sampler.stop() if rank == 0 else {}
     c1 = cache.ff_cache_counters()
     launches = c1["kernel_launches"] - c0["kernel_launches"]
+    choice = cache.ff_cache_kernel_choice()
+    attn_kernel = (f"attn_pair_kernel<false> on CTA pairs" if choice["cta_pair"] > choice["one_cta"]
+                   else f"attn_tcgen05_kernel<{w.head_dim}, false, false>") + f" (+ attn_combine_kernel<{w.head_dim}, false>)"
     st, word = cache.ff_cache_status(stream)
     assert st == 0 and word == 0, (st, hex(word))
 
@@ -921,7 +924,7 @@ def run_gpu(args):
                   h2d_bytes_per_step=3 * call_bytes * n_calls, d2h_bytes_per_step=call_bytes * n_calls,
                   steps=args.e2e_steps, ms_per_step=e2e_ms / args.e2e_steps) if e2e_ms else None),
         gpu_launches=launches,
-        roofline=dict(bound="tensor", kernel=f"attn_tcgen05_kernel<{w.head_dim}, false, false> (+ attn_combine_kernel<{w.head_dim}, false>)",
+        roofline=dict(bound="tensor", kernel=attn_kernel, kernel_launches_by_choice=choice,
                       achieved=attn_tflops, peak=peaks["sustained"],
                       unit="TFLOP/s", frac=attn_tflops / peaks["sustained"], frac_of_burst_peak=attn_tflops / peaks["burst"],
                       peak_source=f"{peaks['source']} bf16 GEMM, sustained (kernel timed inside a long step)",

@@ -44,9 +44,12 @@ enum { FF_BF16 = 0, FF_F32 = 1 };
 
 /* Which attention kernel serves ff_chunk_forward_attn. */
 enum {
-    FF_ATTN_AUTO = 0,    /* tensor-core kernel for FF_BF16 with head_dim 64 or 128, CUDA-core kernel otherwise */
-    FF_ATTN_TCGEN05 = 1, /* TMA + tcgen05/TMEM flash attention (FF_BF16 only) */
-    FF_ATTN_SIMT = 2     /* fp32 CUDA-core flash attention: FF_F32 caches, and an on-device cross-check */
+    FF_ATTN_AUTO = 0,    /* a tensor-core kernel for FF_BF16 with head_dim 64 or 128 (with head_dim 128 the library
+                            picks, per launch, between the two below), the CUDA-core kernel otherwise */
+    FF_ATTN_TCGEN05 = 1, /* TMA + tcgen05/TMEM flash attention, one CTA per SM (FF_BF16 only) */
+    FF_ATTN_SIMT = 2,    /* fp32 CUDA-core flash attention: FF_F32 caches, and an on-device cross-check */
+    FF_ATTN_TCGEN05_PAIR = 3 /* the same attention on CTA pairs (tcgen05 cta_group::2: the two SMs of a TPC share
+                            every K/V tile, each staging half of it); FF_BF16, head_dim 128 only */
 };
 
 typedef struct ff_cache ff_cache; /* opaque HOST object */
@@ -271,6 +274,9 @@ ff_status ff_cache_status(ff_cache* c, void* stream, uint32_t* word /*HOST out*/
 /* Counters since creation/reset: layer-calls, Tail_H advances, anchor publishes, kernels launched. */
 ff_status ff_cache_counters(const ff_cache* c, int64_t* layer_calls, int64_t* advances, int64_t* anchor_publishes,
                             int64_t* kernel_launches);
+/* Attention launches since creation/reset by tensor-core kernel: the one-CTA-per-SM kernel and the kernel on CTA
+ * pairs (see FF_ATTN_AUTO: with head_dim 128 the choice is made per launch). */
+ff_status ff_cache_kernel_choice(const ff_cache* c, int64_t* one_cta_launches, int64_t* cta_pair_launches);
 /* Per-kernel timing for roofline reports.  After ff_cache_profile_begin every layer-call records CUDA events
  * on its stream before the publish kernel, between the two kernels and after the attention kernel (at most
  * max_calls layer-calls are recorded; later ones run untimed; a batched call counts as one record, its publish
@@ -283,11 +289,14 @@ ff_status ff_cache_profile_begin(ff_cache* c, int32_t max_calls);
 ff_status ff_cache_profile_end(ff_cache* c, void* stream, double* publish_ms, int64_t* publish_launches,
                                double* attn_ms, int64_t* attn_launches);
 /* Test hook, HOST only, no device work: enumerates the work distribution of the tensor-core attention kernel for
- * a launch of n_items layer-calls with n_q[i] query rows and n_kv[i] visible keys.  records: cap x 8 int32 (cta,
- * item, head, pair, first key tile, end key tile, scratch slot or -1, second query tile present); header: CTAs,
- * whole pairs per CTA, remainder pairs to merge, iterations per CTA.  Returns the number of pieces, or -1. */
+ * a launch of n_items layer-calls with n_q[i] query rows and n_kv[i] visible keys.  unit_pairs = 1: the kernel
+ * with one CTA per SM (a work unit is one pair of query tiles, a schedule slot one CTA); 2: the kernel on CTA
+ * pairs (a unit is two consecutive pairs, one per CTA of the pair; a slot is a CTA pair, n_ctas_max counts pairs).
+ * records: cap x 8 int32 (slot, item, head, unit, first key tile, end key tile, scratch slot or -1, second query
+ * tile present (one-pair units)); header: slots, whole units per slot, remainder units to merge, iterations per
+ * slot.  Returns the number of pieces, or -1. */
 int32_t ff_debug_schedule(int32_t n_heads, int32_t n_items, const int32_t* n_q, const int32_t* n_kv, int32_t n_ctas_max,
-                          int32_t* records, int32_t cap, int32_t header[4]);
+                          int32_t unit_pairs, int32_t* records, int32_t cap, int32_t header[4]);
 /* Tracing hook: the tensor-core attention kernel appends (event id << 48 | SM clock) records of its first CTA
  * to buf, a caller-owned DEVICE buffer of 3 * cap 64-bit words (softmax group 0, softmax group 1, MMA issuer;
  * cap records each, later events are dropped).  buf = NULL switches tracing off.  Event ids: softmax 1 = waits

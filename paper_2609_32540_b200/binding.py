@@ -13,7 +13,7 @@ from . import build as _build
 
 FF_OK, FF_ERR_INVALID_ARG, FF_ERR_STATE, FF_ERR_OOM, FF_ERR_UNSUPPORTED, FF_ERR_CUDA, FF_ERR_TIMEOUT = range(7)
 FF_BF16, FF_F32 = 0, 1
-FF_ATTN_AUTO, FF_ATTN_TCGEN05, FF_ATTN_SIMT = 0, 1, 2
+FF_ATTN_AUTO, FF_ATTN_TCGEN05, FF_ATTN_SIMT, FF_ATTN_TCGEN05_PAIR = 0, 1, 2, 3
 FF_DEVICE_NONE = -1
 
 _STATUS_NAMES = ["FF_OK", "FF_ERR_INVALID_ARG", "FF_ERR_STATE", "FF_ERR_OOM", "FF_ERR_UNSUPPORTED", "FF_ERR_CUDA",
@@ -26,7 +26,7 @@ SYMBOLS = [
     "ff_sched_run_chunk_host", "ff_sched_run_node", "ff_plan_anchor_count", "ff_plan_anchor_position",
     "ff_plan_window", "ff_cache_profile_begin", "ff_cache_profile_end",
     "ff_cache_ring_state", "ff_cache_anchor_state", "ff_cache_slot_ptr", "ff_cache_status",
-    "ff_cache_counters", "ff_debug_wait_probe", "ff_debug_fail_launch", "ff_debug_set_trace", "ff_chunk_attn_static", "ff_cache_set_qk_gain",
+    "ff_cache_counters", "ff_cache_kernel_choice", "ff_debug_wait_probe", "ff_debug_fail_launch", "ff_debug_set_trace", "ff_chunk_attn_static", "ff_cache_set_qk_gain",
     "ff_euler_step", "ff_plan_sigma", "ff_batch_forward_attn", "ff_sched_run_round", "ff_debug_schedule", "ff_last_cuda_error", "ff_version",
 ]
 
@@ -103,6 +103,7 @@ def load():
     L.ff_cache_slot_ptr.argtypes = [vp, i32, i32, i32, i32, C.POINTER(vp), C.POINTER(vp), i64p, i32p]
     L.ff_cache_status.argtypes = [vp, vp, C.POINTER(C.c_uint32)]
     L.ff_cache_counters.argtypes = [vp, i64p, i64p, i64p, i64p]
+    L.ff_cache_kernel_choice.argtypes = [vp, i64p, i64p]
     L.ff_debug_wait_probe.argtypes = [vp, C.c_uint64, vp]
     L.ff_debug_fail_launch.argtypes = [vp, i32]
     L.ff_debug_set_trace.argtypes = [vp, vp, i32]
@@ -112,7 +113,7 @@ def load():
     L.ff_plan_sigma.argtypes = [i32, i32, C.c_double, C.POINTER(C.c_double)]
     L.ff_batch_forward_attn.argtypes = [vp, i32, C.POINTER(ff_batch_item), i32, vp]
     L.ff_sched_run_round.argtypes = [vp, C.POINTER(ff_round_node), i32, vp]
-    L.ff_debug_schedule.argtypes = [i32, i32, i32p, i32p, i32, i32p, i32, i32p]
+    L.ff_debug_schedule.argtypes = [i32, i32, i32p, i32p, i32, i32, i32p, i32, i32p]
     L.ff_last_cuda_error.restype = i32
     L.ff_version.restype = C.c_char_p
     for name in SYMBOLS:
@@ -293,6 +294,11 @@ class Cache:
                "ff_cache_counters")
         return dict(layer_calls=a.value, advances=b.value, anchor_publishes=c_.value, kernel_launches=d.value)
 
+    def ff_cache_kernel_choice(self) -> dict:
+        a, b = C.c_int64(), C.c_int64()
+        _check(load().ff_cache_kernel_choice(self._h, C.byref(a), C.byref(b)), "ff_cache_kernel_choice")
+        return dict(one_cta=a.value, cta_pair=b.value)
+
     def ff_debug_set_trace(self, buf_ptr, cap) -> int:
         return load().ff_debug_set_trace(self._h, buf_ptr, cap)
 
@@ -346,16 +352,17 @@ def ff_plan_sigma(k, n_stages, shift=5.0) -> float:
     return s.value
 
 
-def ff_debug_schedule(n_heads, n_q, n_kv, n_ctas_max=148):
-    """Host-only: (header dict, list of piece tuples) of the tensor-core kernel's work distribution."""
+def ff_debug_schedule(n_heads, n_q, n_kv, n_ctas_max=148, unit_pairs=1):
+    """Host-only: (header dict, list of piece tuples) of a tensor-core kernel's work distribution (unit_pairs = 2:
+    the kernel on CTA pairs, n_ctas_max then counts pairs)."""
     n = len(n_q)
     aq, ak = (C.c_int32 * n)(*n_q), (C.c_int32 * n)(*n_kv)
     hdr = (C.c_int32 * 4)()
-    total = load().ff_debug_schedule(n_heads, n, aq, ak, n_ctas_max, None, 0, hdr)
+    total = load().ff_debug_schedule(n_heads, n, aq, ak, n_ctas_max, unit_pairs, None, 0, hdr)
     if total < 0:
         raise FFError(FF_ERR_INVALID_ARG, "ff_debug_schedule")
     rec = (C.c_int32 * (8 * max(total, 1)))()
-    load().ff_debug_schedule(n_heads, n, aq, ak, n_ctas_max, rec, total, hdr)
+    load().ff_debug_schedule(n_heads, n, aq, ak, n_ctas_max, unit_pairs, rec, total, hdr)
     pieces = [tuple(rec[8 * i:8 * i + 8]) for i in range(total)]
     return dict(n_ctas=hdr[0], n_full=hdr[1], merge_pairs=hdr[2], iters_per_cta=hdr[3]), pieces
 

@@ -8,7 +8,7 @@ import sys
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libff_chunk_attn.so")
-SOURCES = ["ff_host.cu", "rope_publish.cu", "attn_simt.cu", "attn_sm100.cu", "ff_static.cu", "euler_step.cu"]
+SOURCES = ["ff_host.cu", "rope_publish.cu", "attn_simt.cu", "attn_sm100.cu", "attn_sm100_pair.cu", "ff_static.cu", "euler_step.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]
 

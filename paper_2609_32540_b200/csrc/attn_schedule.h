@@ -2,7 +2,9 @@
 // host-side planner (and enumerable on the host, so that tests can check the cover without a GPU).
 //
 // A launch serves n_items layer-calls.  The unit of work is a pair of 128-row query tiles of one head of one
-// item; pairs are numbered item-major, then head, then pair.  Every CTA first takes n_full whole pairs
+// item (or, for the kernel that runs on CTA pairs, two consecutive pairs of a head: one pair per CTA, both CTAs
+// walking the same key tiles); units are numbered item-major, then head, then unit.  "Pair" below reads "unit"
+// and "CTA" reads "CTA pair" in that case.  Every CTA first takes n_full whole pairs
 // (pair r * n_ctas + cta: the CTAs walk the key tiles of neighbouring pairs in step, so a K/V tile that several
 // of them need is fetched from HBM once and then hit in L2), then an equal share of the (pair, key tile)
 // iterations of the remaining pairs, flattened in pair order; a share may cut pairs, and the pieces of a cut
@@ -91,9 +93,9 @@ struct PieceIter {
             it += p.j1 - p.j0;
         }
         const AttnItem& I = item_at<kTable>(a, p.item);
-        p.h = local / I.n_qp;
-        p.pr = local - p.h * I.n_qp;
-        p.two = 2 * p.pr + 1 < I.n_qt;
+        p.h = local / I.n_up;
+        p.pr = local - p.h * I.n_up;           // unit index inside the head (= pair index when a unit is one pair)
+        p.two = 2 * p.pr + 1 < I.n_qt;         // meaningful for one-pair units only
         return true;
     }
 };

@@ -33,101 +33,9 @@
 //
 // Every wait is bounded (mbar_wait): on expiry an error code goes to the status word and the CTA runs on to
 // its end, frees its tensor memory and returns.
-#include "ff_internal.h"
-#include "attn_schedule.h"
-#include "sm100_ptx.cuh"
+#include "attn_common.cuh"
 
 namespace ffk {
-
-constexpr int kThreads = 384;  // warps 0-7 softmax, 8 producer, 9-10 MMA issuers, 11 idle (fills the warpgroup)
-constexpr uint32_t kTmemCols = 512;
-constexpr int kHalf = 64;   // keys per score buffer: 64 = a 128-key tile is consumed as two halves, 128 = whole tiles
-constexpr int kNB = kTile / kHalf;  // score buffers per query tile
-// S_t[b] / P_t[b]: scores of query tile t against half b of the current key tile
-__host__ __device__ constexpr uint32_t col_s(int t, int b) { return static_cast<uint32_t>(t) * 128u + static_cast<uint32_t>(b) * kHalf; }
-__host__ __device__ constexpr uint32_t col_o(int t) { return 256u + static_cast<uint32_t>(t) * 128u; }  // O_t
-constexpr float kRescaleThreshold = 8.0f;  // in log2 units
-// Registers per thread after setmaxnreg: the two softmax warpgroups take what the third one gives up.
-// setmaxnreg.inc blocks until the registers exist, and no bounded wait can rescue a CTA stuck there, so the
-// total must stay clear of the 64K-register file (a request for exactly 65536 never returned).
-constexpr int kRegsSoftmax = 200, kRegsOther = 96;
-static_assert(2 * 128 * kRegsSoftmax + 128 * kRegsOther <= 64 * 1024 - 2048, "setmaxnreg budget exceeds the register file");
-constexpr float kLog2e = 1.4426950408889634f;
-
-template <int D>
-struct SmemLayout {
-    static constexpr int kBoxBytes = 128 * 64 * 2;           // one 128-row x 64-column bf16 box
-    static constexpr int kTileBytes = kBoxBytes * (D / 64);  // 128 x D
-    static constexpr int kQ = 0;                             // two query tiles
-    static constexpr int kK = 2 * kTileBytes;                // two stages
-    static constexpr int kV = 4 * kTileBytes;                // two stages
-    static constexpr int kTotal = 6 * kTileBytes;
-    // requested size: above half of an SM's shared memory, so that exactly one CTA (which takes all 512
-    // tensor-memory columns) is resident per SM
-    static constexpr int kDynamic = (kTotal + 1024) > 120 * 1024 ? (kTotal + 1024) : 120 * 1024;
-};
-
-// Every kPolyEvery-th pair of exponentials is evaluated by exp2_poly2 on the FMA and integer pipes instead of the
-// MUFU unit (0 = none).  The two softmax warps that share a scheduler collide on its MUFU unit (64 exponentials
-// per row and half tile, 4 lanes per clock), so moving a quarter of them away shortens their exp phase; the step
-// runs on the GPU's power cap, where the extra FMA work costs clock: measured on the 480p shape over 20-step runs,
-// 0: 53.4 ms per step, 4: 52.5, 3: 52.8, 2: 53.2.
-#ifndef FF_POLY_EVERY
-#define FF_POLY_EVERY 4
-#endif
-constexpr int kPolyEvery = FF_POLY_EVERY;
-
-__device__ __forceinline__ float fmax3(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-
-__device__ __forceinline__ float ex2_approx(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-// 2^x for two values on the FMA and integer pipes (no MUFU): x = n + f with n = floor(x) obtained by adding
-// 1.5 * 2^23 with rounding toward -inf, 2^f by a cubic on [0,1) (relative error < 1e-4, far below the bf16
-// rounding the result gets), and n added into the exponent field.  Inputs below -126 give (almost) zero.
-__device__ __forceinline__ float2 exp2_poly2(float2 x) {
-    const float kMagic = 12582912.f;  // 1.5 * 2^23
-    x.x = fmaxf(x.x, -126.f);
-    x.y = fmaxf(x.y, -126.f);
-    const float2 xr = __fadd2_rd(x, make_float2(kMagic, kMagic));
-    const float2 n = __fadd2_rn(xr, make_float2(-kMagic, -kMagic));
-    const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
-    float2 p = __ffma2_rn(make_float2(0.0771190f, 0.0771190f), f, make_float2(0.2275643f, 0.2275643f));
-    p = __ffma2_rn(p, f, make_float2(0.6951461f, 0.6951461f));
-    p = __ffma2_rn(p, f, make_float2(1.f, 1.f));
-    float2 r;
-    r.x = __uint_as_float(__float_as_uint(p.x) + (__float_as_uint(xr.x) << 23));
-    r.y = __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(xr.y) << 23));
-    return r;
-}
-
-// Position in the list of key tiles: segment and token offset inside it.
-struct TileWalker {
-    int seg, t0;
-    __device__ __forceinline__ void seek(const KvSegs& s, int j) {
-        seg = 0;
-        while (seg < s.n) {
-            const int nt = (s.tokens[seg] + kTile - 1) / kTile;
-            if (j < nt) break;
-            j -= nt;
-            ++seg;
-        }
-        t0 = j * kTile;
-    }
-    __device__ __forceinline__ void next(const KvSegs& s) {
-        t0 += kTile;
-        if (t0 >= s.tokens[seg]) { ++seg; t0 = 0; }
-    }
-    __device__ __forceinline__ int row(const KvSegs& s, int h) const { return s.row0[seg] + h * s.head_stride[seg] + t0; }
-    __device__ __forceinline__ int n_valid(const KvSegs& s) const { return min(kTile, s.tokens[seg] - t0); }
-};
 
 // S[128 x 64] = Q_t . (64 keys)^T : D/16 products, both operands K-major in 128-byte-swizzled boxes of 64 columns.
 template <int D>
@@ -523,9 +431,12 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const __grid_constant
     constexpr int kPerLane = D / 32;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     grid_dependency_wait();  // the partial results come from the attention kernel before this launch
-    const long long gr = static_cast<long long>(blockIdx.x) * 8 + warp;  // row index over the remainder pairs
-    const int g = a.n_full * a.n_ctas + static_cast<int>(gr / (2 * kTile));
+    // row index over the remainder units: unit_pairs pairs of 2 x 128 rows each
+    const int up = a.unit_pairs;
+    const long long gr = static_cast<long long>(blockIdx.x) * 8 + warp;
+    const int g = a.n_full * a.n_ctas + static_cast<int>(gr / (up * 2 * kTile));
     if (g >= a.n_pairs) return;
+    const int which = static_cast<int>(gr / (2 * kTile)) % up;   // which pair of the unit (the CTA of a CTA pair that owned it)
     const int rr = static_cast<int>(gr % (2 * kTile));
     const long long cz = a.iters_per_cta;
     int it_i;
@@ -534,12 +445,12 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const __grid_constant
     const long long e_g = s_g + item.n_kv_tiles;
     const int first = static_cast<int>(s_g / cz);
     const int last = static_cast<int>((e_g - 1) / cz);
-    if (first == last) return;  // the pair was handled by one CTA, which stored the final result itself
+    if (first == last) return;  // the unit was handled by one schedule slot, which stored the final result itself
     const int local = g - item.pair0;
-    const int h = local / item.n_qp, pr = local - h * item.n_qp;
+    const int h = local / item.n_up, pr = (local - h * item.n_up) * up + which;
     const int t = rr / kTile, r = rr - t * kTile;
     const int row = (2 * pr + t) * kTile + r;
-    if (2 * pr + t >= item.n_qt || row >= item.n_q) return;
+    if (pr >= item.n_qp || 2 * pr + t >= item.n_qt || row >= item.n_q) return;
     float acc[kPerLane];
 #pragma unroll
     for (int e = 0; e < kPerLane; ++e) acc[e] = 0.f;
@@ -548,7 +459,7 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const __grid_constant
         // a CTA's piece of this pair sits in scratch slot 2*cta when the CTA's share begins inside the pair
         // (then it was the CTA's first piece), else in slot 2*cta + 1
         const long long c0 = static_cast<long long>(cta) * cz;
-        const int slot = 2 * cta + ((c0 >= s_g && c0 < e_g) ? 0 : 1);
+        const int slot = 2 * (cta * up + which) + ((c0 >= s_g && c0 < e_g) ? 0 : 1);
         const size_t prow = (static_cast<size_t>(slot) * 2 + t) * kTile + r;
         const float2 ml = a.part_ml[prow];
         const float* po = a.part_o + prow * D + lane * kPerLane;
@@ -604,12 +515,13 @@ static int plan_impl(AttnArgs& a, AttnItem* items, int n_ctas_max) {
         AttnItem& I = items[i];
         I.n_qt = (I.n_q + kTile - 1) / kTile;
         I.n_qp = (I.n_qt + 1) / 2;
+        I.n_up = (I.n_qp + a.unit_pairs - 1) / a.unit_pairs;
         int tiles = 0;
         for (int s = 0; s < I.segs.n; ++s) tiles += (I.segs.tokens[s] + kTile - 1) / kTile;
         I.n_kv_tiles = tiles;
         I.pair0 = static_cast<int>(n_pairs);
-        n_pairs += static_cast<long long>(a.n_heads) * I.n_qp;
-        work += static_cast<long long>(a.n_heads) * I.n_qp * tiles;
+        n_pairs += static_cast<long long>(a.n_heads) * I.n_up;
+        work += static_cast<long long>(a.n_heads) * I.n_up * tiles;
     }
     a.n_pairs = static_cast<int>(n_pairs);
     long long n_cta = work / 4;  // at least four key tiles per CTA
@@ -621,7 +533,7 @@ static int plan_impl(AttnArgs& a, AttnItem* items, int n_ctas_max) {
     long long iters = 0;
     for (int i = 0; i < a.n_items; ++i) {
         AttnItem& I = items[i];
-        const long long pairs = static_cast<long long>(a.n_heads) * I.n_qp;
+        const long long pairs = static_cast<long long>(a.n_heads) * I.n_up;
         long long first_rem = g0 - I.pair0;
         if (first_rem < 0) first_rem = 0;
         if (first_rem > pairs) first_rem = pairs;
@@ -641,6 +553,7 @@ static int plan_impl(AttnArgs& a, AttnItem* items, int n_ctas_max) {
 }
 
 int attn_tcgen05_plan(AttnArgs& a, AttnItem* items, int n_ctas_max) {
+    if (a.unit_pairs < 1) a.unit_pairs = 1;
     if (items == a.items) {
         a.items_tab = nullptr;
         return plan_impl<false>(a, items, n_ctas_max);
@@ -655,10 +568,11 @@ template <int D>
 static cudaError_t launch_impl(const AttnArgs& a, int merge_pairs, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                                const CUtensorMap& tm_v, cudaStream_t s) {
     const bool table = a.items_tab != nullptr, trace = a.trace != nullptr && !table;
-    const dim3 grid(a.n_ctas), block(kThreads), mgrid(merge_pairs * (2 * kTile / 8)), mblock(256);
+    const dim3 grid(a.n_ctas), block(kThreads), mgrid(merge_pairs * a.unit_pairs * (2 * kTile / 8)), mblock(256);
     const size_t smem = SmemLayout<D>::kDynamic;
     cudaError_t e;
-    if (table) e = launch_overlapped(attn_tcgen05_kernel<D, false, true>, grid, block, smem, s, tm_q, tm_k, tm_v, a);
+    if (a.unit_pairs == 2) e = launch_attn_pair(a, tm_q, tm_k, tm_v, s);   // tm_k: the map with 32-row boxes
+    else if (table) e = launch_overlapped(attn_tcgen05_kernel<D, false, true>, grid, block, smem, s, tm_q, tm_k, tm_v, a);
     else if (trace) e = launch_overlapped(attn_tcgen05_kernel<D, true, false>, grid, block, smem, s, tm_q, tm_k, tm_v, a);
     else e = launch_overlapped(attn_tcgen05_kernel<D, false, false>, grid, block, smem, s, tm_q, tm_k, tm_v, a);
     if (e == cudaSuccess && merge_pairs)

@@ -11,6 +11,12 @@
 #include "ff_internal.h"
 #include "attn_schedule.h"
 
+// What FF_ATTN_AUTO does with head_dim 128: 1 = choose per launch between the kernel on CTA pairs (cta_group::2)
+// and the one-CTA-per-SM kernel, 0 = always the latter.
+#ifndef FF_CTA_PAIR_DEFAULT
+#define FF_CTA_PAIR_DEFAULT 1
+#endif
+
 using namespace ffk;
 
 namespace {
@@ -35,7 +41,7 @@ struct Derived {
     int32_t R;  // slots per bank: H + 1 unless the caller asked for more (several chunks of one stage per launch)
     int64_t ring_rows, anchor_rows, total_rows;
     size_t off_tab_f, off_tab_y, off_tab_x, off_status, off_items, off_gain, off_k, off_v, off_q, off_part_o, off_part_ml, off_stage, stage_bytes, total;
-    int impl;
+    int impl, pair_mode;
 };
 
 ff_status derive(const ff_cache_config* cfg, Derived* D) {
@@ -56,7 +62,16 @@ ff_status derive(const ff_cache_config* cfg, Derived* D) {
     static_assert(FF_MAX_BATCH == kMaxBatch, "ff.h and ff_internal.h disagree on the batch limit");
     if (cfg->head_dim != 64 && cfg->head_dim != 128) return FF_ERR_UNSUPPORTED;
     int impl = cfg->attn_impl;
-    if (impl == FF_ATTN_AUTO) impl = cfg->dtype == FF_BF16 ? FF_ATTN_TCGEN05 : FF_ATTN_SIMT;
+    // pair_mode: 0 = one-CTA-per-SM kernel, 1 = CTA-pair kernel, 2 = chosen per launch
+    D->pair_mode = 0;
+    if (impl == FF_ATTN_AUTO) {
+        impl = cfg->dtype == FF_BF16 ? FF_ATTN_TCGEN05 : FF_ATTN_SIMT;
+        if (impl == FF_ATTN_TCGEN05 && cfg->head_dim == 128 && FF_CTA_PAIR_DEFAULT) D->pair_mode = 2;
+    } else if (impl == FF_ATTN_TCGEN05_PAIR) {
+        if (cfg->head_dim != 128) return FF_ERR_UNSUPPORTED;
+        impl = FF_ATTN_TCGEN05;
+        D->pair_mode = 1;
+    }
     if (impl != FF_ATTN_TCGEN05 && impl != FF_ATTN_SIMT) return FF_ERR_INVALID_ARG;
     if (impl == FF_ATTN_TCGEN05 && cfg->dtype != FF_BF16) return FF_ERR_UNSUPPORTED;
     D->impl = impl;
@@ -126,6 +141,8 @@ struct ff_cache {
     std::vector<int32_t> anchor_pos;               // per anchor slot
     std::vector<uint8_t> anchor_valid;             // [slot][layer]
     CUtensorMap tm_q, tm_k, tm_v;
+    CUtensorMap tm_k32;               // K in boxes of 32 rows (the kernel on CTA pairs stages a quarter tile per copy)
+    int pair_slots = 0;               // CTA pairs that can be resident at once; 0 = the pair kernel is not used
     int64_t n_layer_calls = 0, n_advances = 0, n_anchor_publishes = 0, n_launches = 0;
     std::vector<cudaEvent_t> prof_events;  // 3 per recorded layer-call
     size_t prof_used = 0;
@@ -144,6 +161,7 @@ struct ff_cache {
     uint32_t launch_seq = 0;        // numbers the attention launches; tags the error codes a launch records
     int32_t fail_launch_in = 0;     // test hook: the n-th launch site from now reports a failure without launching
     int64_t prof_publish_launches = 0, prof_attn_launches = 0;
+    int64_t n_attn_single = 0, n_attn_pair = 0;   // attention launches by tensor-core kernel
 
     SlotMeta& slot(int stage, int layer, int s) {
         return slots[((size_t)stage * cfg.n_layers + layer) * D.R + s];
@@ -192,6 +210,7 @@ void reset_meta(ff_cache* c) {
     std::fill(c->anchor_pos.begin(), c->anchor_pos.end(), -1);
     std::fill(c->anchor_valid.begin(), c->anchor_valid.end(), 0);
     c->n_layer_calls = c->n_advances = c->n_anchor_publishes = c->n_launches = 0;
+    c->n_attn_single = c->n_attn_pair = 0;
 }
 
 // Rotary tables: angle = pos * theta^(-j/n) in double, cos and sin in double, each rounded once to float.
@@ -205,10 +224,10 @@ void fill_table(std::vector<float2>& tab, int n_pos, int n_pairs, double theta) 
         }
 }
 
-bool make_map(EncodeTiledFn enc, CUtensorMap* m, void* base, int64_t rows, int d) {
+bool make_map(EncodeTiledFn enc, CUtensorMap* m, void* base, int64_t rows, int d, int box_rows = kTile) {
     cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)d * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     cuuint32_t es[2] = {1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -331,6 +350,18 @@ ff_status ff_cache_create(const ff_cache_config* cfg, void* arena, size_t arena_
             return FF_ERR_CUDA;
         }
         if (!cuda_ok(attn_tcgen05_prepare(D.d))) { delete c; return FF_ERR_CUDA; }
+        if (D.pair_mode != 0) {
+            int pairs = 0;
+            if (!make_map(enc, &c->tm_k32, c->arena + D.off_k, D.total_rows, D.d, 32) || !cuda_ok(attn_pair_prepare(&pairs))) {
+                delete c;
+                return FF_ERR_CUDA;
+            }
+            c->pair_slots = pairs < kMaxCtas / 2 ? pairs : kMaxCtas / 2;
+            if (c->pair_slots < 1) {
+                if (D.pair_mode == 1) { delete c; return FF_ERR_UNSUPPORTED; }
+                c->D.pair_mode = 0;
+            }
+        }
     }
     *out = c;
     return FF_OK;
@@ -607,7 +638,25 @@ ff_status forward_batch(ff_cache* c, int32_t layer, const CallDesc* d, int32_t n
         it.segs.n = m;
     }
     const bool tc = c->D.impl == FF_ATTN_TCGEN05;
-    const int merge_pairs = tc ? attn_tcgen05_plan(a, items, c->sm_count < kMaxCtas ? c->sm_count : kMaxCtas) : 0;
+    // Which tensor-core kernel: the CTA-pair kernel moves half the K/V bytes per query row into shared memory and is
+    // about 6 % faster per (unit, key tile) step, but its units are four query tiles where the other kernel's are
+    // two, so a head whose tile count is 1 mod 4 leaves more of its last unit empty.  Chosen per launch from the
+    // query-tile slots each kernel would spend (measured: 720p, 85 tiles per head, +5 %; 480p, 37 tiles, a tie).
+    bool pair = tc && c->D.pair_mode == 1;
+    if (tc && c->D.pair_mode == 2 && !c->trace) {
+        long long slots_single = 0, slots_pair = 0;
+        for (int i = 0; i < n; ++i) {
+            const long long n_qt = (items[i].n_q + kTile - 1) / kTile;
+            long long tiles = 0;
+            for (int sg = 0; sg < items[i].segs.n; ++sg) tiles += (items[i].segs.tokens[sg] + kTile - 1) / kTile;
+            slots_single += (n_qt + 1) / 2 * 2 * tiles;
+            slots_pair += (n_qt + 3) / 4 * 4 * tiles;
+        }
+        pair = slots_pair * 100 <= slots_single * 104;
+    }
+    a.unit_pairs = pair ? 2 : 1;
+    const int merge_pairs = !tc ? 0 : pair ? attn_tcgen05_plan(a, items, c->pair_slots > 0 ? c->pair_slots : 74)
+                                           : attn_tcgen05_plan(a, items, c->sm_count < kMaxCtas ? c->sm_count : kMaxCtas);
 
     int64_t launched = 0, pub_launches = 0, attn_launches = 0;
     if (ev) cudaEventRecord(ev[0], s);
@@ -633,7 +682,7 @@ ff_status forward_batch(ff_cache* c, int32_t layer, const CallDesc* d, int32_t n
                 a.items_tab = dev_tab;
             }
             int nl = 1;
-            if (!cuda_ok(launch_attn_tcgen05(a, merge_pairs, c->tm_q, c->tm_k, c->tm_v, s, &nl))) return FF_ERR_CUDA;
+            if (!cuda_ok(launch_attn_tcgen05(a, merge_pairs, c->tm_q, pair ? c->tm_k32 : c->tm_k, c->tm_v, s, &nl))) return FF_ERR_CUDA;
             attn_launches += nl;
         } else {
             attn_launches += merge_pairs ? 2 : 1;
@@ -655,6 +704,7 @@ ff_status forward_batch(ff_cache* c, int32_t layer, const CallDesc* d, int32_t n
         m.n_tokens = pend[i].n_tokens;
     }
     ++c->launch_seq;
+    if (tc) ++(pair ? c->n_attn_pair : c->n_attn_single);
     if (ev) {
         c->prof_used += 3;
         c->prof_publish_launches += pub_launches;
@@ -902,19 +952,28 @@ ff_status ff_cache_counters(const ff_cache* c, int64_t* layer_calls, int64_t* ad
     return FF_OK;
 }
 
+ff_status ff_cache_kernel_choice(const ff_cache* c, int64_t* one_cta_launches, int64_t* cta_pair_launches) {
+    if (!c) return FF_ERR_INVALID_ARG;
+    if (one_cta_launches) *one_cta_launches = c->n_attn_single;
+    if (cta_pair_launches) *cta_pair_launches = c->n_attn_pair;
+    return FF_OK;
+}
+
 /* Test hook, host only: the work distribution the tensor-core kernel would use for a launch of n_items
  * layer-calls with n_q[i] query rows and n_kv[i] visible keys (taken as one segment each).  Writes up to cap
  * records of 8 int32 (cta, item, head, pair, first key tile, end key tile, scratch slot or -1, second tile
  * present) in the order each CTA walks them and returns the total number of records (which may exceed cap);
  * header[0..3] = CTAs, whole pairs per CTA, remainder pairs to merge (0 = none), iterations per CTA. */
 int32_t ff_debug_schedule(int32_t n_heads, int32_t n_items, const int32_t* n_q, const int32_t* n_kv, int32_t n_ctas_max,
-                          int32_t* records, int32_t cap, int32_t header[4]) {
+                          int32_t unit_pairs, int32_t* records, int32_t cap, int32_t header[4]) {
+    if (unit_pairs != 1 && unit_pairs != 2) return -1;
     if (n_heads < 1 || n_items < 1 || n_items > kMaxBatch || !n_q || !n_kv || n_ctas_max < 1 || n_ctas_max > kMaxCtas ||
         cap < 0 || (cap > 0 && !records))
         return -1;
     AttnArgs a{};
     a.n_heads = n_heads;
     a.n_items = n_items;
+    a.unit_pairs = unit_pairs;
     std::vector<AttnItem> tab(n_items > kMaxInline ? n_items : 0);
     AttnItem* items = n_items > kMaxInline ? tab.data() : a.items;
     for (int i = 0; i < n_items; ++i) {

@@ -64,6 +64,7 @@ struct AttnItem {
     int32_t n_q;
     // schedule of the tensor-core kernel (filled by attn_tcgen05_plan)
     int32_t n_qt, n_qp;   // query tiles and query-tile pairs per head
+    int32_t n_up;         // work units per head: a unit is one pair (single-CTA kernel) or two consecutive pairs (CTA-pair kernel)
     int32_t n_kv_tiles;   // key tiles over all visible segments
     int32_t pair0;        // index of the item's first pair in the launch-wide order (item, head, pair)
     int32_t rem_pair0;    // first pair of the item (item-local index) that lies in the cut remainder
@@ -89,10 +90,11 @@ struct AttnArgs {
     const AttnItem* items_tab;  // n_items > kMaxInline: the descriptors (device memory; host memory while planning)
     AttnItem items[kMaxInline]; // n_items <= kMaxInline: the descriptors themselves
     // schedule of the tensor-core kernel (filled by attn_tcgen05_plan)
-    int32_t n_pairs;          // query-tile pairs over all items and heads
+    int32_t unit_pairs;       // pairs per work unit: 1 (single-CTA kernel) or 2 (CTA-pair kernel: one pair per CTA)
+    int32_t n_pairs;          // work units over all items and heads (pairs, when unit_pairs == 1)
     int32_t n_full;           // whole pairs every CTA handles first (pair r * n_ctas + cta)
     int32_t iters_per_cta;    // share of the remaining pairs' (pair, key tile) iterations per CTA
-    int32_t n_ctas;
+    int32_t n_ctas;           // schedule slots: CTAs (single-CTA kernel) or CTA pairs
     long long total_iters;    // (pair, key tile) iterations of the remaining pairs
     float* part_o;            // [slot][2][128][d] unnormalised accumulators of split pairs
     float2* part_ml;          // [slot][2][128]    (reference maximum in log2 units, row sum)
@@ -139,6 +141,11 @@ int attn_tcgen05_plan(AttnArgs& a, AttnItem* items, int n_ctas_max);
 cudaError_t launch_attn_tcgen05(const AttnArgs& a, int merge_pairs, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                                 const CUtensorMap& tm_v, cudaStream_t s, int* n_launches);
 cudaError_t attn_tcgen05_prepare(int head_dim);  // sets the dynamic shared-memory attribute once
+// The kernel on CTA pairs (head_dim 128): prepare reports how many pairs can be resident at once; launch takes a
+// planned `a` with unit_pairs == 2, n_ctas = CTA pairs, and the K map whose boxes hold 32 rows.
+cudaError_t attn_pair_prepare(int* max_pairs);
+cudaError_t launch_attn_pair(const AttnArgs& a, const CUtensorMap& tm_q, const CUtensorMap& tm_k32, const CUtensorMap& tm_v,
+                             cudaStream_t s);
 cudaError_t launch_wait_probe(uint32_t* status, unsigned long long limit_ns, cudaStream_t s);
 
 }  // namespace ffk

@@ -27,11 +27,22 @@ def test_wan1p3b_480p_full_shape():
     gpu.close()
 
 
+@pytest.mark.parametrize("name,frames,layer", [("wan1p3b_480p", 12, 1), ("wan1p3b_720p", 9, 0)])
+def test_cta_pair_kernel_at_full_token_counts(name, frames, layer):
+    """The kernel on CTA pairs (cta_group::2), forced: 480p (37 query tiles per head: the last unit of a head holds
+    one tile of four) and 720p (85 tiles), warm-up and steady-state chunks, sampled rows and published slots."""
+    w = W.scaled(W.CONFIGS[name], total_frames=frames, n_layers=2)
+    stats, gpu, orc = Hn.run_both(w, O.BF16, attn_impl=3, seed=12, rows_fn=rows_fn, check_layers=[layer],
+                                  check_stages=[0, 2], pooled=True)
+    assert len(stats) == (frames // 3) * 2
+    gpu.close()
+
+
 def test_wan1p3b_480p_every_row_of_a_steady_state_call():
     """One steady-state layer-call of config 2 (anchor + two history chunks + own chunk: 15600 keys) compared with
     the oracle on ALL 4680 rows x 12 heads, not a sample: about half a minute of CPU work for the oracle."""
     w = W.scaled(W.CONFIGS["wan1p3b_480p"], total_frames=9, n_layers=1)
-    stats, gpu, orc = Hn.run_both(w, O.BF16, attn_impl=1, seed=11, rows_fn=None, check_layers=[0], check_stages=[1],
+    stats, gpu, orc = Hn.run_both(w, O.BF16, attn_impl=0, seed=11, rows_fn=None, check_layers=[0], check_stages=[1],
                                   pooled=True, check_chunks=[2])
     assert len(stats) == 1 and stats[0]["max_abs"] > 0
     gpu.close()
@@ -49,7 +60,7 @@ def test_wan1p3b_480p_peaked_logits():
 def test_wan1p3b_720p_full_shape():
     """Config 4: 10800 query tokens, two anchor frames, N_kv up to 39600."""
     w = W.scaled(W.CONFIGS["wan1p3b_720p"], total_frames=12)
-    stats, gpu, orc = Hn.run_both(w, O.BF16, attn_impl=1, seed=5, rows_fn=rows_fn, check_layers=[17],
+    stats, gpu, orc = Hn.run_both(w, O.BF16, attn_impl=0, seed=5, rows_fn=rows_fn, check_layers=[17],
                                   check_stages=[1], pooled=True, check_chunks=[0, 3])
     assert len(stats) == 2
     gpu.close()
@@ -60,7 +71,7 @@ def test_wan14b_720p_full_shape():
     w = W.scaled(W.CONFIGS["wan14b_720p_stream35s"], total_frames=9)
     free, total = torch.cuda.mem_get_info()
     assert free > 130e9, f"needs about 120 GB of free device memory, have {free / 1e9:.0f} GB"
-    stats, gpu, orc = Hn.run_both(w, O.BF16, attn_impl=1, seed=6, rows_fn=lambda n: W.sample_rows(n, extra=2),
+    stats, gpu, orc = Hn.run_both(w, O.BF16, attn_impl=0, seed=6, rows_fn=lambda n: W.sample_rows(n, extra=2),
                                   check_layers=[39], check_stages=[3], pooled=True, check_chunks=[0, 2])
     assert len(stats) == 2
     gpu.close()

@@ -109,6 +109,19 @@ def test_whole_clip_in_one_launch_tiny_and_ragged():
     gpu.close()
 
 
+def test_cta_pair_kernel_in_batched_launches():
+    """The kernel on CTA pairs under the two batched forms: wavefront rounds (four nodes per launch, ragged shapes,
+    a short last chunk) and a whole clip in one launch (descriptor table)."""
+    w = W.Workload("pair_wavefront", 2, 3, 128, 9, 23, 2, 4, 2, 11, 2, 6, "bracket", 4)
+    stats, gpu, orc = Hn.run_wavefront(w, O.BF16, attn_impl=3, seed=6, rows_fn=lambda n: W.sample_rows(n, 16, 6))
+    assert len(stats) == w.n_chunks * w.n_stages * w.n_layers
+    gpu.close()
+    w = W.Workload("pair_clip", 2, 3, 128, 9, 23, 2, 2, 2, 19, 2, 6, "bracket", 4)
+    stats, gpu, orc = Hn.run_packed_clip(w, w.n_chunks, O.BF16, attn_impl=3, seed=7, rows_fn=lambda n: W.sample_rows(n, 16, 7))
+    assert len(stats) == w.n_chunks * w.n_stages * w.n_layers
+    gpu.close()
+
+
 def test_whole_81_latent_clip_in_one_launch_at_480p_token_counts():
     """The paper's worked example at full 480p token counts (27 chunks, H = 5, three anchors per window), one stage
     and two layers: ONE attention launch per layer over all 27 chunks; sampled rows of every chunk against the

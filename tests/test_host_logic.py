@@ -193,18 +193,20 @@ def test_qk_norm_option_validation_and_arena_growth(B):
     c.close()
 
 
-def _check_schedule(B, n_heads, n_q, n_kv, n_ctas_max=148):
-    hdr, pieces = B.ff_debug_schedule(n_heads, n_q, n_kv, n_ctas_max)
+def _check_schedule(B, n_heads, n_q, n_kv, n_ctas_max=148, unit_pairs=1):
+    """unit_pairs = 2: the kernel on CTA pairs; a unit is two consecutive pairs of query tiles, a slot a CTA pair."""
+    hdr, pieces = B.ff_debug_schedule(n_heads, n_q, n_kv, n_ctas_max, unit_pairs)
     tiles = [-(-k // 128) for k in n_kv]
     n_qt = [-(-q // 128) for q in n_q]
-    n_qp = [(t + 1) // 2 for t in n_qt]
+    n_qp = [-(-((t + 1) // 2) // unit_pairs) for t in n_qt]     # units per head
     cover = {}
     per_cta = {}
     slots_seen = set()
     for cta, item, h, pr, j0, j1, slot, two in pieces:
         assert 0 <= item < len(n_q) and 0 <= h < n_heads and 0 <= pr < n_qp[item]
         assert 0 <= j0 < j1 <= tiles[item]
-        assert bool(two) == (2 * pr + 1 < n_qt[item])
+        if unit_pairs == 1:
+            assert bool(two) == (2 * pr + 1 < n_qt[item])
         whole = j0 == 0 and j1 == tiles[item]
         if whole:
             assert slot == -1
@@ -265,6 +267,8 @@ def _check_schedule(B, n_heads, n_q, n_kv, n_ctas_max=148):
 def test_attention_work_distribution_covers_everything_once(B, n_heads, n_q, n_kv):
     for n_ctas in (148, 7, 1):
         _check_schedule(B, n_heads, n_q, n_kv, n_ctas)
+    for n_pairs_of_ctas in (74, 5, 1):
+        _check_schedule(B, n_heads, n_q, n_kv, n_pairs_of_ctas, unit_pairs=2)
 
 
 def test_same_stage_batches_follow_the_slot_rule(B):
