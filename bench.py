@@ -35,8 +35,9 @@ WORKLOAD = "wan1p3b_480p"
 NOMINAL_BF16_TFLOPS = 2250.0
 N_IO = 8                 # distinct resident Q/K/V sets cycled over the layer-calls (345 MB > the 126 MB L2)
 CPU_SAMPLE_ROWS = 0      # query rows of one steady-state layer-call the oracle is timed on (0 = all of them)
-ATTN_KERNEL_SOURCE = os.path.join(ROOT, "paper_2609_32540_b200", "csrc", "attn_sm100.cu")
-ATTN_PROFILE = os.path.join(ROOT, "profiles", "attn_tcgen05_wan1p3b_480p.json")
+# committed ncu summaries of the dominant kernel, by workload (each names the kernel source it was captured from)
+ATTN_PROFILES = {"wan1p3b_480p": os.path.join(ROOT, "profiles", "attn_tcgen05_wan1p3b_480p.json"),
+                 "wan1p3b_720p": os.path.join(ROOT, "profiles", "attn_pair_wan1p3b_720p.json")}
 
 
 def blob_hash(path: str) -> str:
@@ -47,15 +48,17 @@ def blob_hash(path: str) -> str:
 
 
 def ncu_traffic(workload: str) -> dict:
-    """DRAM bytes per attention launch from the committed ncu summary of the headline workload, with a flag that
-    says whether the kernel source has changed since that capture (then the figure describes an older kernel)."""
-    if workload != WORKLOAD or not os.path.exists(ATTN_PROFILE):
+    """DRAM bytes per attention launch from the committed ncu summary of this workload, with a flag that says
+    whether the kernel's source has changed since that capture (then the figure describes an older kernel)."""
+    path = ATTN_PROFILES.get(workload)
+    if path is None or not os.path.exists(path):
         return dict(traffic=None, traffic_source="no ncu capture of this workload")
-    prof = json.load(open(ATTN_PROFILE))
+    prof = json.load(open(path))
     per_launch = prof["dram_bytes_read_per_launch"] + prof["dram_bytes_write_per_launch"]
-    return dict(traffic=per_launch, traffic_source=os.path.relpath(ATTN_PROFILE, ROOT),
-                traffic_stale=blob_hash(ATTN_KERNEL_SOURCE) != prof["kernel_source_blob"],
-                traffic_captured_on=prof.get("capture_case"))
+    return dict(traffic=per_launch, traffic_source=os.path.relpath(path, ROOT), traffic_kernel=prof["kernel"],
+                traffic_stale=blob_hash(os.path.join(ROOT, prof["kernel_source"])) != prof["kernel_source_blob"],
+                traffic_captured_on=prof.get("capture_case"),
+                tensor_pipe_active_pct_in_capture=prof.get("sm_pipe_tensor_cycles_active_pct_elapsed"))
 
 
 def read_peaks():
