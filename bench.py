@@ -40,11 +40,14 @@ ATTN_PROFILES = {"wan1p3b_480p": os.path.join(ROOT, "profiles", "attn_tcgen05_wa
                  "wan1p3b_720p": os.path.join(ROOT, "profiles", "attn_pair_wan1p3b_720p.json")}
 
 
-def blob_hash(path: str) -> str:
-    """The hash git gives a file's content (sha1 over a "blob <size>" header and the bytes)."""
+def blob_hash(paths) -> str:
+    """One hash over the contents of the files (in the given order): sha1 of their git blob hashes."""
     import hashlib
-    data = open(path, "rb").read()
-    return hashlib.sha1(b"blob %d\0" % len(data) + data).hexdigest()
+    h = hashlib.sha1()
+    for path in paths:
+        data = open(os.path.join(ROOT, path), "rb").read()
+        h.update(hashlib.sha1(b"blob %d\0" % len(data) + data).hexdigest().encode())
+    return h.hexdigest()
 
 
 def ncu_traffic(workload: str) -> dict:
@@ -56,7 +59,7 @@ def ncu_traffic(workload: str) -> dict:
     prof = json.load(open(path))
     per_launch = prof["dram_bytes_read_per_launch"] + prof["dram_bytes_write_per_launch"]
     return dict(traffic=per_launch, traffic_source=os.path.relpath(path, ROOT), traffic_kernel=prof["kernel"],
-                traffic_stale=blob_hash(os.path.join(ROOT, prof["kernel_source"])) != prof["kernel_source_blob"],
+                traffic_stale=blob_hash(prof["kernel_sources"]) != prof["kernel_sources_hash"],
                 traffic_captured_on=prof.get("capture_case"),
                 tensor_pipe_active_pct_in_capture=prof.get("sm_pipe_tensor_cycles_active_pct_elapsed"))
 

@@ -18,8 +18,17 @@ constexpr float kRescaleThreshold = 8.0f;  // in log2 units
 // Registers per thread after setmaxnreg: the two softmax warpgroups take what the third one gives up.
 // setmaxnreg.inc blocks until the registers exist, and no bounded wait can rescue a CTA stuck there, so the
 // total must stay clear of the 64K-register file (a request for exactly 65536 never returned).
-constexpr int kRegsSoftmax = 200, kRegsOther = 96;
-static_assert(2 * 128 * kRegsSoftmax + 128 * kRegsOther <= 64 * 1024 - 2048, "setmaxnreg budget exceeds the register file");
+// The split also steers the compiler's register allocation in the softmax loop, and more is not better: measured
+// per 480p layer-call on the one-CTA kernel, softmax/other = 160..216: 200/96 0.402 ms, 216/64 0.408, 208/80 0.413,
+// 192/112 0.408, 184/128 0.398, 176/144 0.403, 168/160 0.404; on the CTA-pair kernel at 720p 200/96 2.090 ms,
+// 184/128 2.114, 176/144 2.082.
+template <int kSoftmax, int kOther>
+struct RegSplit {
+    static constexpr int softmax = kSoftmax, other = kOther;
+    static_assert(2 * 128 * kSoftmax + 128 * kOther <= 64 * 1024 - 2048, "setmaxnreg budget exceeds the register file");
+};
+using RegsOneCta = RegSplit<184, 128>;
+using RegsCtaPair = RegSplit<176, 144>;
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int D>

@@ -123,7 +123,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     grid_dependency_wait();
 
     if (warp >= 8) {
-      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(RegsOneCta::other));
       if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -268,7 +268,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
       }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(RegsOneCta::softmax));
         // ------------------------------------------------------------------ softmax + epilogue (one row per thread)
         const int t = warp >> 2;                                   // query tile of the pair this group serves
         const int r = threadIdx.x & 127;                           // row inside the tile

@@ -110,7 +110,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     grid_dependency_wait();
 
     if (warp >= 8) {
-      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(RegsCtaPair::other));
       if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer (one lane, in each CTA)
         if (lane == 0) {
@@ -239,7 +239,7 @@ attn_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         }
       }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(RegsCtaPair::softmax));
         // ------------------------------------------------------------------ softmax + epilogue (one row per thread),
         // in both CTAs, each on its own 128 rows of the pair's products
         const int t = warp >> 2;

@@ -221,6 +221,31 @@ def test_expired_device_wait_is_reported_and_the_context_stays_usable():
     gpu.close()
 
 
+def test_auto_kernel_choice_follows_the_query_tile_count():
+    """FF_ATTN_AUTO with head_dim 128: the kernel on CTA pairs when four-tile units waste at most 4 % more query-tile
+    slots than two-tile units (8 tiles per head: none; 5 tiles: 8 slots against 6), the one-CTA kernel otherwise;
+    forcing a kernel is honoured; head_dim 64 has only the one-CTA kernel."""
+    from paper_2609_32540_b200 import binding as B
+    cases = [(8 * 128, 0, "cta_pair"), (5 * 128, 0, "one_cta"), (8 * 128, 1, "one_cta"), (5 * 128, 3, "cta_pair")]
+    for n_tok, impl, want in cases:
+        w = W.Workload("choice", 1, 2, 128, 8, n_tok // 8, 1, 1, 0, 1, 0, 0, "none", 1)
+        gpu = Hn.GpuCache(w, O.BF16, attn_impl=impl)
+        q, k, v = (t.cuda() for t in W.qkv(w, 0, 0, 0, 0, 1))
+        st, out = gpu.forward(0, 0, 0, 1, 0, q, k, v, [])
+        assert st == 0
+        torch.cuda.synchronize()
+        c = gpu.cache.ff_cache_kernel_choice()
+        assert c[want] == 1 and c["one_cta" if want == "cta_pair" else "cta_pair"] == 0, (n_tok, impl, c)
+        orc = Hn.make_oracle(w, O.BF16)
+        so, truth = orc.chunk_forward(0, 0, 0, 1, 0, q.float().cpu().numpy(), k.float().cpu().numpy(), v.float().cpu().numpy(), [])
+        Hn.compare_outputs(out, truth, O.BF16, f"kernel choice {n_tok} {impl}")
+        gpu.close()
+    w64 = W.scaled(W.CONFIGS["tiny"], anchor_policy="none", n_anchor_slots=0)
+    with pytest.raises(B.FFError) as e:
+        Hn.GpuCache(w64, O.BF16, attn_impl=3)
+    assert e.value.status == B.FF_ERR_UNSUPPORTED
+
+
 def test_profile_hooks_time_both_kernels():
     w = W.CONFIGS["tiny"]
     gpu = Hn.GpuCache(w, O.BF16, 1)
