@@ -93,16 +93,24 @@ __device__ __forceinline__ void inv_rms_shared(float (&acc)[4], int ppr, float i
     for (int i = 0; i < 4; ++i) acc[i] = __shfl_sync(0xffffffffu, inv, row_lane0 + i);
 }
 template <int E>
-__device__ __forceinline__ void scale_row(float (&x)[E], const float (&gain)[E], float inv) {
+__device__ __forceinline__ void scale_row(float (&x)[E], const float* __restrict__ gain, float inv) {
+    // the thread's E channel gains are read where they are used (two 16-byte loads that hit L1): holding them in
+    // registers for the whole kernel cost a resident block per SM
 #pragma unroll
-    for (int e = 0; e < E; ++e) x[e] = __fmul_rn(__fmul_rn(x[e], inv), gain[e]);
+    for (int e = 0; e < E; e += 4) {
+        const float4 g = __ldg(reinterpret_cast<const float4*>(gain + e));
+        x[e] = __fmul_rn(__fmul_rn(x[e], inv), g.x);
+        x[e + 1] = __fmul_rn(__fmul_rn(x[e + 1], inv), g.y);
+        x[e + 2] = __fmul_rn(__fmul_rn(x[e + 2], inv), g.z);
+        x[e + 3] = __fmul_rn(__fmul_rn(x[e + 3], inv), g.w);
+    }
 }
 
 // Thread layout: a thread keeps one 16-byte piece position of the (token, head) row for the whole kernel, so the
 // rotary pairs it handles - and with them the table and axis each pair reads - are fixed; it walks over the
 // rows of its block's contiguous share with 32-bit index arithmetic.  Q and K share the cos/sin values.
 template <bool kBf16, bool kNorm>
-__global__ void __launch_bounds__(256) rope_publish_kernel(const __grid_constant__ PublishBatch batch) {
+__global__ void __launch_bounds__(256, kNorm ? 3 : 0) rope_publish_kernel(const __grid_constant__ PublishBatch batch) {
     const PublishArgs& a = batch.items[blockIdx.y];
     constexpr int kElemsPerPiece = kBf16 ? 8 : 4;
     constexpr int kPairs = kElemsPerPiece / 2;
@@ -134,12 +142,8 @@ __global__ void __launch_bounds__(256) rope_publish_kernel(const __grid_constant
         }
     }
     // the gains of this thread's channels (its piece position never changes)
-    float gain_q[kElemsPerPiece], gain_k[kElemsPerPiece];
-#pragma unroll
-    for (int e = 0; e < kElemsPerPiece; ++e) {
-        gain_q[e] = kNorm ? __ldg(a.gain_q + piece * kElemsPerPiece + e) : 1.0f;
-        gain_k[e] = kNorm ? __ldg(a.gain_k + piece * kElemsPerPiece + e) : 1.0f;
-    }
+    const float* gain_q = kNorm ? a.gain_q + piece * kElemsPerPiece : nullptr;
+    const float* gain_k = kNorm ? a.gain_k + piece * kElemsPerPiece : nullptr;
     const uint4* __restrict__ qin = reinterpret_cast<const uint4*>(a.q);
     const uint4* __restrict__ kin = reinterpret_cast<const uint4*>(a.k);
     const uint4* __restrict__ vin = reinterpret_cast<const uint4*>(a.v);
