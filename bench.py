@@ -984,14 +984,21 @@ def main():
     ap.add_argument("--stream", action="store_true",
                     help="extra: also run the workload's whole stream once from empty banks and report its wall time")
     ap.add_argument("--skip-extra", action="store_true", help="skip the extra measurement at the paper's budget")
-    ap.add_argument("--mode", default="replicas", choices=["replicas", "wavefront"],
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "wavefront", "adjacent"],
                     help="replicas (default, the headline): every rank runs the whole path on its own GPU; wavefront: "
-                         "the paper's stage-per-GPU pipeline over --gpus ranks (1, 2 or 4 for four stages)")
+                         "the paper's stage-per-GPU pipeline over --gpus ranks (1, 2 or 4 for four stages); adjacent: "
+                         "only the extra timings of the publish pass with and without q/k normalisation and of the "
+                         "Euler update (one GPU; the small case the publish kernels are profiled on)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
     elif args.mode == "wavefront":
         run_wavefront_mode(args)
+    elif args.mode == "adjacent":
+        import paper_2609_32540_b200 as P
+        torch.cuda.set_device(0)
+        print(json.dumps(dict(mode="adjacent", adjacent_steps=measure_adjacent_steps(
+            P, torch.device("cuda:0"), 0, read_peaks()["hbm_gbs"]))), flush=True)
     else:
         run_gpu(args)
 

@@ -9,6 +9,8 @@
 // the result can be checked bit for bit.
 #include <cuda_bf16.h>
 
+#include <atomic>
+
 #include "../../include/ff.h"
 #include "ff_internal.h"
 
@@ -43,6 +45,7 @@ __global__ void __launch_bounds__(256) euler_step_kernel(const void* x_, const v
     XT* out = static_cast<XT*>(out_);
     const long long n_vec = n / kVec;
     const long long stride = (long long)gridDim.x * blockDim.x;
+    ffk::grid_dependency_wait();  // launched as a programmatic dependent: x and v may come from the kernel before
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += stride) {
         alignas(16) XT xs[kVec];
         alignas(16) VT vs[kVec];
@@ -77,9 +80,15 @@ extern "C" ff_status ff_euler_step(const void* x, const void* v, float sigma_k, 
         return FF_ERR_INVALID_ARG;
     if (((uintptr_t)x | (uintptr_t)v | (uintptr_t)out) & 15u) return FF_ERR_INVALID_ARG;
     if (n == 0) return FF_OK;
-    int device = 0, sms = 148;
+    // the SM count of each device is asked once (the call is a large part of the host time of a launch this small)
+    static std::atomic<int> sms_of[64];
+    int device = 0;
     if (cudaGetDevice(&device) != cudaSuccess) return FF_ERR_CUDA;
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    int sms = (device >= 0 && device < 64) ? sms_of[device].load(std::memory_order_relaxed) : 0;
+    if (sms == 0) {
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 1) sms = 148;
+        if (device >= 0 && device < 64) sms_of[device].store(sms, std::memory_order_relaxed);
+    }
     const long long n_vec = n / 8;
     long long blocks = (n_vec + 255) / 256;
     const long long cap = (long long)sms * 8;  // a whole number of waves of 8 resident blocks per SM
@@ -88,11 +97,16 @@ extern "C" ff_status ff_euler_step(const void* x, const void* v, float sigma_k, 
     const float dsigma = sigma_k - sigma_km1;  // rounded once, on the host, in float
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool xb = dtype_x == FF_BF16, vb = dtype_v == FF_BF16;
-    if (xb && vb) euler_step_kernel<true, true><<<(unsigned)blocks, 256, 0, s>>>(x, v, out, n, dsigma);
-    else if (xb) euler_step_kernel<true, false><<<(unsigned)blocks, 256, 0, s>>>(x, v, out, n, dsigma);
-    else if (vb) euler_step_kernel<false, true><<<(unsigned)blocks, 256, 0, s>>>(x, v, out, n, dsigma);
-    else euler_step_kernel<false, false><<<(unsigned)blocks, 256, 0, s>>>(x, v, out, n, dsigma);
-    return cudaGetLastError() == cudaSuccess ? FF_OK : FF_ERR_CUDA;
+    // One chunk's latent is a few hundred thousand elements: the launch itself is most of the cost, so the grid is
+    // set up under the tail of the kernel before it in the stream, like the library's other kernels.
+    const dim3 grid((unsigned)blocks), block(256);
+    const long long nn = n;
+    cudaError_t e;
+    if (xb && vb) e = ffk::launch_overlapped(euler_step_kernel<true, true>, grid, block, 0, s, x, v, out, nn, dsigma);
+    else if (xb) e = ffk::launch_overlapped(euler_step_kernel<true, false>, grid, block, 0, s, x, v, out, nn, dsigma);
+    else if (vb) e = ffk::launch_overlapped(euler_step_kernel<false, true>, grid, block, 0, s, x, v, out, nn, dsigma);
+    else e = ffk::launch_overlapped(euler_step_kernel<false, false>, grid, block, 0, s, x, v, out, nn, dsigma);
+    return e == cudaSuccess ? FF_OK : FF_ERR_CUDA;
 }
 
 // sigma_k = shift * u / (1 + (shift - 1) * u) with u = k / S: the uniform levels 1, (S-1)/S, ..., 1/S, 0 pushed

@@ -110,7 +110,7 @@ __device__ __forceinline__ void scale_row(float (&x)[E], const float* __restrict
 // rotary pairs it handles - and with them the table and axis each pair reads - are fixed; it walks over the
 // rows of its block's contiguous share with 32-bit index arithmetic.  Q and K share the cos/sin values.
 template <bool kBf16, bool kNorm>
-__global__ void __launch_bounds__(256, kNorm ? 3 : 0) rope_publish_kernel(const __grid_constant__ PublishBatch batch) {
+__global__ void __launch_bounds__(256, kNorm ? 2 : 0) rope_publish_kernel(const __grid_constant__ PublishBatch batch) {
     const PublishArgs& a = batch.items[blockIdx.y];
     constexpr int kElemsPerPiece = kBf16 ? 8 : 4;
     constexpr int kPairs = kElemsPerPiece / 2;
@@ -155,6 +155,25 @@ __global__ void __launch_bounds__(256, kNorm ? 3 : 0) rope_publish_kernel(const 
     // The loop bound is the same for all threads of a warp (the normalisation shuffles across a row's threads).
     const int first_row = row_begin + rowslot;
     const int n_iter = (row_end - row_begin + 2 * rows_per_pass - 1) / (2 * rows_per_pass);
+    // With the normalisation the loads of iteration it+1 are issued before the arithmetic of iteration it (all
+    // blocks start together and walk in step: without that the memory system idles while everybody reduces).
+    uint4 nk[kNorm ? 2 : 1], nv[kNorm ? 2 : 1], nq[kNorm ? 2 : 1];
+    auto fetch_ahead = [&](int it) {
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int row = first_row + (2 * it + u) * rows_per_pass;
+            nk[u] = nv[u] = nq[u] = make_uint4(0, 0, 0, 0);
+            if (row < n_rows && row < row_end) {
+                const long long src = (long long)row * ppr + piece;
+                nk[u] = __ldg(kin + src);
+                nv[u] = __ldg(vin + src);
+                if (qin) nq[u] = __ldg(qin + src);
+            }
+        }
+    };
+    if constexpr (kNorm) {
+        if (n_iter > 0) fetch_ahead(0);
+    }
     for (int it = 0; it < n_iter; ++it) {
         const int row0 = first_row + it * 2 * rows_per_pass;
         uint4 kv[2], vv[2], qv[2];
@@ -167,12 +186,16 @@ __global__ void __launch_bounds__(256, kNorm ? 3 : 0) rope_publish_kernel(const 
             data[u] = row < n_rows && live[u];
             tt[u] = row / a.n_heads;
             hh[u] = row - tt[u] * a.n_heads;
-            kv[u] = vv[u] = qv[u] = make_uint4(0, 0, 0, 0);
-            if (data[u]) {
-                const long long src = (long long)row * ppr + piece;
-                kv[u] = __ldg(kin + src);
-                vv[u] = __ldg(vin + src);
-                if (qin) qv[u] = __ldg(qin + src);
+            if constexpr (kNorm) {
+                kv[u] = nk[u]; vv[u] = nv[u]; qv[u] = nq[u];
+            } else {
+                kv[u] = vv[u] = qv[u] = make_uint4(0, 0, 0, 0);
+                if (data[u]) {
+                    const long long src = (long long)row * ppr + piece;
+                    kv[u] = __ldg(kin + src);
+                    vv[u] = __ldg(vin + src);
+                    if (qin) qv[u] = __ldg(qin + src);
+                }
             }
         }
         // with the normalisation both rows are unpacked and normalised first (their inverse RMS values are evaluated
@@ -184,6 +207,7 @@ __global__ void __launch_bounds__(256, kNorm ? 3 : 0) rope_publish_kernel(const 
                 unpack_piece<kBf16>(kv[u], kxs[u]);
                 unpack_piece<kBf16>(qv[u], qxs[u]);
             }
+            if (it + 1 < n_iter) fetch_ahead(it + 1);
             float acc[4];
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
