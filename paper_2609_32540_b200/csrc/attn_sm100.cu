@@ -302,68 +302,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     for (int q2 = 0; q2 < kHalf / 32; ++q2) tmem_ld_32x32b_x32(tmem + lane_addr + col_s(t, b) + q2 * 32, sr[q2]);
                     tmem_ld_wait();
                     tr.mark(3);
-                    if (n_here < kHalf) {
-#pragma unroll
-                        for (int q2 = 0; q2 < kHalf / 32; ++q2)
-#pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (q2 * 32 + i >= n_here) sr[q2][i] = 0xff800000u;  // -inf
-                    }
-                    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-                    for (int q2 = 0; q2 < kHalf / 32; ++q2)
-#pragma unroll
-                        for (int i = 0; i < 32; i += 2)
-                            mx[(i >> 1) & 3] = fmax3(mx[(i >> 1) & 3], __uint_as_float(sr[q2][i]),
-                                                     __uint_as_float(sr[q2][i + 1]));
-                    const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-
-                    // raise the reference maximum only when some row of this warp outgrew it by the threshold
-                    const bool grow = (tmax - m_used) * c > kRescaleThreshold;  // true on the first half (m_used = -inf)
-                    if (__any_sync(0xffffffffu, grow)) {
-                        const float m_new = fmaxf(m_used, tmax);
-                        if (j > p.j0 || b > 0) {
-                            // O_t may only be touched once the product fed by the previous half tile has finished
-                            mbar_wait(&bar_pv_done[t], (halves - 1) & 1, a.status, a.launch_tag | kErrWaitO);
-                            tc_fence_after_sync();
-                            const float alpha = ex2_approx((m_used - m_new) * c);
-                            l *= alpha;
-#pragma unroll
-                            for (int q4 = 0; q4 < D / 32; ++q4) {
-                                uint32_t o[32];
-                                tmem_ld_32x32b_x32(tmem + lane_addr + col_o(t) + q4 * 32, o);
-                                tmem_ld_wait();
-#pragma unroll
-                                for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                                tmem_st_32x32b_x32(tmem + lane_addr + col_o(t) + q4 * 32, o);
-                            }
-                            tmem_st_wait();
-                        }
-                        m_used = m_new;
-                    }
-                    const float2 c2 = make_float2(c, c);
-                    const float2 nmc2 = make_float2(-m_used * c, -m_used * c);
-                    float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll
-                    for (int q2 = 0; q2 < kHalf / 32; ++q2) {
-                        uint32_t pk[16];
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const float2 x = __ffma2_rn(
-                                make_float2(__uint_as_float(sr[q2][2 * i]), __uint_as_float(sr[q2][2 * i + 1])), c2, nmc2);
-                            float2 pr;
-                            if (kPolyEvery > 0 && (i % (kPolyEvery > 0 ? kPolyEvery : 1)) == 0) {
-                                pr = exp2_poly2(x);   // a fraction of the exponentials on the FMA pipe
-                            } else {
-                                pr.x = ex2_approx(x.x);
-                                pr.y = ex2_approx(x.y);
-                            }
-                            sum2[i & 1] = __fadd2_rn(sum2[i & 1], pr);
-                            pk[i] = pack_bf16x2(pr.x, pr.y);
-                        }
-                        tmem_st_32x32b_x16(tmem + lane_addr + col_s(t, b) + q2 * 16, pk);
-                    }
-                    l += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
+                    softmax_half_step<D>(sr, n_here, c, j == p.j0 && b == 0, tmem + lane_addr + col_s(t, b),
+                                         tmem + lane_addr + col_o(t), &bar_pv_done[t], (halves - 1) & 1, a.status,
+                                         a.launch_tag | kErrWaitO, m_used, l);
                     tr.mark(4);
                     tmem_st_wait();
                     tr.mark(5);
