@@ -51,10 +51,8 @@ __device__ __forceinline__ uint4 rotate_pack_piece(const float (&x)[kBf16 ? 8 : 
         for (int i = 0; i < 4; ++i) {
             float r0, r1;
             rotate(x[2 * i], x[2 * i + 1], cs[i], r0, r1);
-            __nv_bfloat162 o;
-            o.x = __float2bfloat16_rn(r0);
-            o.y = __float2bfloat16_rn(r1);
-            w[i] = *reinterpret_cast<uint32_t*>(&o);
+            const __nv_bfloat162 o = __floats2bfloat162_rn(r0, r1);  // one conversion for the pair, each half RNE
+            w[i] = *reinterpret_cast<const uint32_t*>(&o);
         }
     } else {
         float r0, r1, r2, r3;
@@ -105,6 +103,33 @@ __device__ __forceinline__ void scale_row(float (&x)[E], const float* __restrict
         x[e + 3] = __fmul_rn(__fmul_rn(x[e + 3], inv), g.w);
     }
 }
+
+// Where a (token, head) row sits: token t = (f, py, px) on the chunk's grid, head h.  A thread's rows advance by a
+// fixed number of rows per iteration, so the position is carried along (one set of divisions per thread at the
+// start) instead of being recomputed with four integer divisions per row.
+struct RowPos {
+    int row, t, h, f, py, px;
+    __device__ __forceinline__ void init(int row_, int n_heads, int grid_w, int tf) {
+        row = row_;
+        t = row / n_heads;
+        h = row - t * n_heads;
+        f = t / tf;
+        const int r = t - f * tf;
+        py = r / grid_w;
+        px = r - py * grid_w;
+    }
+    // row += step, with step = dt * n_heads + dh, 0 <= dh < n_heads
+    __device__ __forceinline__ void advance(int step, int dt, int dh, int n_heads, int grid_h, int grid_w) {
+        row += step;
+        h += dh;
+        int inc = dt;
+        if (h >= n_heads) { h -= n_heads; ++inc; }
+        t += inc;
+        px += inc;
+        while (px >= grid_w) { px -= grid_w; ++py; }
+        while (py >= grid_h) { py -= grid_h; ++f; }
+    }
+};
 
 // Thread layout: a thread keeps one 16-byte piece position of the (token, head) row for the whole kernel, so the
 // rotary pairs it handles - and with them the table and axis each pair reads - are fixed; it walks over the
@@ -174,18 +199,22 @@ __global__ void __launch_bounds__(256, kNorm ? 2 : 0) rope_publish_kernel(const 
     if constexpr (kNorm) {
         if (n_iter > 0) fetch_ahead(0);
     }
+    RowPos next_row;   // the first of the two rows of the coming iteration
+    next_row.init(first_row, a.n_heads, a.grid_w, tf);
+    const int half_dt = rows_per_pass / a.n_heads, half_dh = rows_per_pass - half_dt * a.n_heads;
     for (int it = 0; it < n_iter; ++it) {
-        const int row0 = first_row + it * 2 * rows_per_pass;
+        RowPos at[2];
+        at[0] = next_row;
+        next_row.advance(rows_per_pass, half_dt, half_dh, a.n_heads, a.grid_h, a.grid_w);
+        at[1] = next_row;
+        next_row.advance(rows_per_pass, half_dt, half_dh, a.n_heads, a.grid_h, a.grid_w);
         uint4 kv[2], vv[2], qv[2];
-        int tt[2], hh[2];
         bool live[2], data[2];
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
-            const int row = row0 + u * rows_per_pass;
+            const int row = at[u].row;
             live[u] = row < row_end;
             data[u] = row < n_rows && live[u];
-            tt[u] = row / a.n_heads;
-            hh[u] = row - tt[u] * a.n_heads;
             if constexpr (kNorm) {
                 kv[u] = nk[u]; vv[u] = nv[u]; qv[u] = nq[u];
             } else {
@@ -229,14 +258,13 @@ __global__ void __launch_bounds__(256, kNorm ? 2 : 0) rope_publish_kernel(const 
                 unpack_piece<kBf16>(kv[u], kx);
                 unpack_piece<kBf16>(qv[u], qx);
             }
+            const RowPos& here = at[u];
             if (!live[u]) continue;
-            const int t = tt[u], h = hh[u];
+            const int t = here.t, h = here.h;
             const long long dst = ((long long)a.dst_row0 + (long long)h * a.dst_head_stride + t) * ppr + piece;
             const long long qdst = ((long long)h * a.q_rows_per_head + t) * ppr + piece;
             if (data[u]) {
-                const int f = t / tf, r = t - f * tf;
-                const int py = r / a.grid_w, px = r - py * a.grid_w;
-                const int pos[3] = {a.first_frame_pos + f * a.frame_pos_stride, py, px};
+                const int pos[3] = {a.first_frame_pos + here.f * a.frame_pos_stride, here.py, here.px};
                 float2 cs[4];
 #pragma unroll
                 for (int i = 0; i < kPairs; ++i) cs[i] = __ldg(tab[i] + pos[axis[i]] * tab_stride[i]);
