@@ -373,17 +373,20 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     grid_dependency_wait();  // the partial results come from the attention kernel before this launch
     // row index over the remainder units: unit_pairs pairs of 2 x 128 rows each
+    // (32-bit arithmetic throughout: the launcher only starts this kernel when the row count and the iteration
+    // count of the remainder fit, and a 64-bit division costs a warp this short a third of its instructions)
     const int up = a.unit_pairs;
-    const long long gr = static_cast<long long>(blockIdx.x) * 8 + warp;
-    const int g = a.n_full * a.n_ctas + static_cast<int>(gr / (up * 2 * kTile));
+    const uint32_t gr = blockIdx.x * 8u + static_cast<uint32_t>(warp);
+    const uint32_t pair_of_row = gr / (2 * kTile);                  // 2 * kTile is a power of two
+    const int g = a.n_full * a.n_ctas + static_cast<int>(up == 2 ? pair_of_row >> 1 : pair_of_row);
     if (g >= a.n_pairs) return;
-    const int which = static_cast<int>(gr / (2 * kTile)) % up;   // which pair of the unit (the CTA of a CTA pair that owned it)
+    const int which = up == 2 ? static_cast<int>(pair_of_row & 1u) : 0;   // which pair of the unit (the CTA of a CTA pair that owned it)
     const int rr = static_cast<int>(gr % (2 * kTile));
-    const long long cz = a.iters_per_cta;
+    const uint32_t cz = static_cast<uint32_t>(a.iters_per_cta);
     int it_i;
-    const long long s_g = rem_iter_start<kTable>(a, g, &it_i);
+    const uint32_t s_g = static_cast<uint32_t>(rem_iter_start<kTable>(a, g, &it_i));
     const AttnItem& item = item_at<kTable>(a, it_i);
-    const long long e_g = s_g + item.n_kv_tiles;
+    const uint32_t e_g = s_g + static_cast<uint32_t>(item.n_kv_tiles);
     const int first = static_cast<int>(s_g / cz);
     const int last = static_cast<int>((e_g - 1) / cz);
     if (first == last) return;  // the unit was handled by one schedule slot, which stored the final result itself
@@ -399,7 +402,7 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const __grid_constant
     for (int cta = first; cta <= last; ++cta) {
         // a CTA's piece of this pair sits in scratch slot 2*cta when the CTA's share begins inside the pair
         // (then it was the CTA's first piece), else in slot 2*cta + 1
-        const long long c0 = static_cast<long long>(cta) * cz;
+        const uint32_t c0 = static_cast<uint32_t>(cta) * cz;
         const int slot = 2 * (cta * up + which) + ((c0 >= s_g && c0 < e_g) ? 0 : 1);
         const size_t prow = (static_cast<size_t>(slot) * 2 + t) * kTile + r;
         const float2 ml = a.part_ml[prow];
@@ -511,6 +514,7 @@ static cudaError_t launch_impl(const AttnArgs& a, int merge_pairs, const CUtenso
     const bool table = a.items_tab != nullptr, trace = a.trace != nullptr && !table;
     const dim3 grid(a.n_ctas), block(kThreads), mgrid(merge_pairs * a.unit_pairs * (2 * kTile / 8)), mblock(256);
     const size_t smem = SmemLayout<D>::kDynamic;
+    if (merge_pairs && a.total_iters >= (1ll << 31)) return cudaErrorInvalidValue;  // the merge kernel indexes in 32 bits
     cudaError_t e;
     if (a.unit_pairs == 2) e = launch_attn_pair(a, tm_q, tm_k, tm_v, s);   // tm_k: the map with 32-row boxes
     else if (table) e = launch_overlapped(attn_tcgen05_kernel<D, false, true>, grid, block, smem, s, tm_q, tm_k, tm_v, a);
