@@ -57,3 +57,16 @@ def test_random_configuration_in_all_three_schedules(seed):
     stats, gpu, _ = Hn.run_packed_clip(w, group, dtype, attn_impl=impl, seed=seed, rows_fn=rows)
     assert len(stats) == w.n_chunks * w.n_stages * w.n_layers
     gpu.close()
+
+
+@pytest.mark.parametrize("seed", list(range(100, 116)))
+def test_random_configuration_with_the_fused_qk_normalisation(seed):
+    """The same kind of shapes with raw Q/K rows and the normalisation fused into the publish pass (every other
+    seed with per-channel gains): the published cache must still match the oracle bit for bit."""
+    w = _random_workload(seed)
+    rows = None if w.chunk_frames * w.tokens_per_frame <= 400 else (lambda n: W.sample_rows(n, 24, seed))
+    dtype, impl = (O.F32, 2) if seed % 5 == 4 else (O.BF16, 3 if w.head_dim == 128 and seed % 2 == 0 else 1)
+    stats, gpu, _ = Hn.run_both(w, dtype, attn_impl=impl, seed=seed, rows_fn=rows, qk_norm_eps=1e-6,
+                                qk_gains=(seed % 2 == 0))
+    assert len(stats) == w.n_chunks * w.n_stages * w.n_layers
+    gpu.close()
