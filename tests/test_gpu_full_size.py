@@ -94,3 +94,23 @@ def test_wan1p3b_480p_long_stream():
         assert s["next_chunk"] == 87 and s["head"] == 87 % 3 and s["count"] == 2
         assert sorted(s["slot_chunk"]) == [84, 85, 86]
     gpu.close()
+
+
+@pytest.mark.parametrize("name,chunks", [("wan1p3b_480p", 5), ("wan1p3b_720p", 4)])
+def test_every_row_at_full_token_counts_agrees_between_the_two_tensor_core_kernels(name, chunks):
+    """An extra next to the sampled-row comparisons with the oracle (CUDA against CUDA, so it pins nothing by
+    itself): over warm-up and steady-state chunks at full token counts, EVERY output row of the kernel with one
+    CTA per SM and of the kernel on CTA pairs is finite and the two agree to a bf16 rounding step.  Their work
+    distributions differ (pairs of tiles against units of four, other cut points), so a row that one of them
+    dropped or merged wrongly cannot hide here."""
+    from tests import test_gpu_api as A
+    base = W.CONFIGS[name]
+    w = W.scaled(base, n_layers=1, n_stages=1, total_frames=chunks * base.chunk_frames)
+    a, ga = A._run(w, "chunk", impl=1)
+    b, gb = A._run(w, "chunk", impl=3)
+    assert len(a) == chunks
+    for key in a:
+        assert torch.isfinite(a[key].float()).all() and torch.isfinite(b[key].float()).all(), key
+        worst = (a[key].float() - b[key].float()).abs().max().item()
+        assert worst <= 2e-3, (key, worst)
+    ga.close(); gb.close()
